@@ -1,0 +1,9 @@
+"""CPU oracle for the masked convolution: test infrastructure, not part of the product.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg import this package.
+It shares no code with the CUDA path and never imports it.
+"""
+from .masked_conv import (build, bf16_round, kept_list, masked_conv, masked_conv_rows,
+                          n_threads)
+
+__all__ = ["build", "bf16_round", "kept_list", "masked_conv", "masked_conv_rows", "n_threads"]

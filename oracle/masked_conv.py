@@ -1,0 +1,129 @@
+"""ctypes wrapper around the plain-C oracle (oracle/masked_conv_oracle.c).
+
+The C file is the oracle; this module only compiles it with gcc (-O2, OpenMP over output
+rows) and marshals numpy arrays.  See the C file's header for what is computed and which
+passages of the paper it follows.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "masked_conv_oracle.c")
+_LIB = os.path.join(_HERE, "libasx_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc if the shared object is missing or stale."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + f".tmp{os.getpid()}"
+    subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-shared", "-fPIC",
+                           "-o", tmp, _SRC])
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i64, i32p = ctypes.c_int64, ctypes.POINTER(ctypes.c_int32)
+        fp, dp, u8p = (ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_double),
+                       ctypes.POINTER(ctypes.c_uint8))
+        i64p = ctypes.POINTER(ctypes.c_int64)
+        ci = ctypes.c_int
+        lib.asxo_bf16_round.argtypes = [fp, fp, i64]
+        lib.asxo_bf16_round.restype = None
+        lib.asxo_kept_list.argtypes = [u8p, i64, i32p]
+        lib.asxo_kept_list.restype = i64
+        conv_args = [fp, ci, ci, ci, ci, fp, ci, ci, ci, ci, ci, fp, u8p, i64, ci]
+        lib.asxo_masked_conv.argtypes = conv_args + [dp]
+        lib.asxo_masked_conv.restype = ci
+        lib.asxo_masked_conv_rows.argtypes = conv_args + [i64p, i64, dp]
+        lib.asxo_masked_conv_rows.restype = ci
+        _lib = lib
+    return _lib
+
+
+def n_threads() -> int:
+    """Threads the OpenMP loops will use (OMP_NUM_THREADS, else all cores)."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    return int(env) if env else (os.cpu_count() or 1)
+
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _ptr(a: np.ndarray, ctype):
+    return a.ctypes.data_as(ctypes.POINTER(ctype))
+
+
+def bf16_round(a) -> np.ndarray:
+    """Round fp32 values to bfloat16 (nearest, ties to even); returned as fp32."""
+    a = _f32(a)
+    out = np.empty_like(a)
+    _load().asxo_bf16_round(_ptr(a, ctypes.c_float), _ptr(out, ctypes.c_float), a.size)
+    return out
+
+
+def kept_list(mask) -> np.ndarray:
+    """Ascending positions with mask == 1, int32."""
+    mask = np.ascontiguousarray(mask, dtype=np.uint8).ravel()
+    kept = np.empty(mask.size, dtype=np.int32)
+    c = _load().asxo_kept_list(_ptr(mask, ctypes.c_uint8), mask.size, _ptr(kept, ctypes.c_int32))
+    return kept[:c].copy()
+
+
+def _geometry(x, w, stride, pad):
+    Nb, H, W, C_in = x.shape
+    C_out, kh, kw, C_in2 = w.shape
+    if C_in != C_in2:
+        raise ValueError("channel mismatch")
+    Ho = (H + 2 * pad - kh) // stride + 1
+    Wo = (W + 2 * pad - kw) // stride + 1
+    return Nb, H, W, C_in, C_out, kh, kw, Ho, Wo
+
+
+def masked_conv(x, w, bias: Optional[np.ndarray], mask, stride: int, pad: int,
+                relu: bool) -> np.ndarray:
+    """y[Nb][Ho][Wo][C_out] in fp64.  x is NHWC fp32, w is [C_out][kh][kw][C_in] fp32 (both are
+    rounded to bf16 inside), bias fp32 or None, mask uint8 of Ho*Wo or Nb*Ho*Wo entries."""
+    x, w = _f32(x), _f32(w)
+    Nb, H, W, C_in, C_out, kh, kw, Ho, Wo = _geometry(x, w, stride, pad)
+    mask = np.ascontiguousarray(mask, dtype=np.uint8).ravel()
+    b = None if bias is None else _f32(bias)
+    y = np.empty((Nb, Ho, Wo, C_out), dtype=np.float64)
+    rc = _load().asxo_masked_conv(
+        _ptr(x, ctypes.c_float), Nb, H, W, C_in, _ptr(w, ctypes.c_float), C_out, kh, kw,
+        stride, pad, None if b is None else _ptr(b, ctypes.c_float),
+        _ptr(mask, ctypes.c_uint8), mask.size, int(bool(relu)), _ptr(y, ctypes.c_double))
+    if rc:
+        raise ValueError(f"oracle rejected the arguments (code {rc})")
+    return y
+
+
+def masked_conv_rows(x, w, bias, mask, stride: int, pad: int, relu: bool, sel) -> np.ndarray:
+    """The same definition at selected lowered rows only: returns [len(sel)][C_out] fp64."""
+    x, w = _f32(x), _f32(w)
+    Nb, H, W, C_in, C_out, kh, kw, Ho, Wo = _geometry(x, w, stride, pad)
+    mask = np.ascontiguousarray(mask, dtype=np.uint8).ravel()
+    b = None if bias is None else _f32(bias)
+    sel = np.ascontiguousarray(sel, dtype=np.int64).ravel()
+    y = np.empty((sel.size, C_out), dtype=np.float64)
+    rc = _load().asxo_masked_conv_rows(
+        _ptr(x, ctypes.c_float), Nb, H, W, C_in, _ptr(w, ctypes.c_float), C_out, kh, kw,
+        stride, pad, None if b is None else _ptr(b, ctypes.c_float),
+        _ptr(mask, ctypes.c_uint8), mask.size, int(bool(relu)),
+        _ptr(sel, ctypes.c_int64), sel.size, _ptr(y, ctypes.c_double))
+    if rc:
+        raise ValueError(f"oracle rejected the arguments (code {rc})")
+    return y
