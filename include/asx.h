@@ -1,0 +1,163 @@
+/*
+ * asx — masked convolution as a compacted GEMM on NVIDIA B200 (sm_100a).
+ *
+ * The library computes the inference path of "Accelerating Deep Neural Networks via
+ * Semi-Structured Activation Sparsity" (arXiv 2309.06626), Section 3.2 and Appendix A
+ * (Algorithm 2): a convolution lowered to a matrix product in which a per-layer binary mask
+ * with one entry per output spatial position removes whole rows of the lowered activation
+ * matrix.  The product runs on the kept rows only; dropped positions are zero in every
+ * channel.  With x[Nb][H][W][C_in] (NHWC), w[C_out][kh][kw][C_in], bias[C_out]:
+ *
+ *     y[n][oy][ox][co] = mask(n,oy,ox) ? act(bias[co] + sum_{ky,kx,ci} x[n][oy*s-p+ky][ox*s-p+kx][ci]
+ *                                                                    * w[co][ky][kx][ci])
+ *                                      : 0
+ *
+ * (cross-correlation, zero padding p on all sides, dilation 1, groups 1).  x, w and y are
+ * bfloat16, the bias is fp32, products are accumulated in fp32 on the tensor cores, and y is
+ * rounded to bfloat16 (nearest even).  A dropped position is the bit pattern 0x0000 in all
+ * channels: neither bias nor activation is applied there.
+ *
+ * Conventions for every function:
+ *  - returns an asx_status; nothing throws or aborts; arguments are checked on the host
+ *    before any launch and a failed check launches nothing;
+ *  - "device pointer" means memory of the current CUDA device, owned by the caller;
+ *  - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream);
+ *    work is enqueued on it and the call returns without waiting unless stated;
+ *  - a layer handle may be used by one host thread at a time;
+ *  - there is no CPU fallback: without a usable CUDA device the calls return ASX_ERR_CUDA.
+ */
+#ifndef ASX_H_
+#define ASX_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct asx_layer asx_layer;   /* opaque, owned by the library */
+
+typedef enum {
+    ASX_OK = 0,
+    ASX_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, unknown flag */
+    ASX_ERR_UNSUPPORTED = 2,   /* a legal convolution this build cannot run */
+    ASX_ERR_NO_MASK = 3,       /* asx_run before any asx_set_mask* */
+    ASX_ERR_SHAPE = 4,         /* mask length does not match the output geometry */
+    ASX_ERR_ALIGN = 5,         /* a pointer is not aligned as documented */
+    ASX_ERR_OOM = 6,           /* device or host allocation failed */
+    ASX_ERR_CUDA = 7,          /* a CUDA runtime or driver call failed */
+    ASX_ERR_TIMEOUT = 8        /* a bounded wait inside a kernel gave up */
+} asx_status;
+
+/* flags of asx_run */
+enum {
+    ASX_ACT_RELU = 1,      /* y = max(acc + bias, 0) on kept rows (default: acc + bias) */
+    ASX_RECOMPACT = 2,     /* rebuild the kept-row list from the stored mask inside this call */
+    ASX_IMPL_NAIVE = 4     /* run the slow one-thread-per-output CUDA kernel (debug reference) */
+};
+
+/* Human-readable name of a status code; never NULL; static storage. */
+const char* asx_status_string(asx_status s);
+
+/*
+ * Create a layer: the convolution geometry of Section 3 (filter size, stride, padding).
+ * C_in, C_out, kh, kw, stride >= 1, pad >= 0.  On success *out receives a handle to be
+ * released with asx_destroy.  No device memory is allocated here.
+ */
+asx_status asx_create_layer(int C_in, int C_out, int kh, int kw, int stride, int pad,
+                            asx_layer** out);
+
+/*
+ * Set the layer's binary mask (Appendix A, Algorithm 2: mask == 1 keeps an output position,
+ * mask == 0 drops it) and build the kept-row list (stage i of Section 3.2, the running index
+ * of the indirection initialisation): kept[j] = position of the j-th non-zero mask entry in
+ * ascending order, index p = oy*Wo + ox.
+ *   mask : `rows` bytes, each 0 or non-zero, host or device pointer (the library finds out
+ *          which); it is copied, the caller may free it after the call returns.
+ *   rows : Ho*Wo (one mask shared by every image of a batch, the paper's constant per-layer
+ *          mask) or Nb*Ho*Wo (one entry per lowered row); checked against the geometry at
+ *          asx_run.  0 < rows < 2^31.
+ * The copy and the compaction kernel are enqueued on `cuda_stream`; a host mask is copied
+ * synchronously.  Device buffers owned by the layer are (re)allocated when `rows` grows.
+ */
+asx_status asx_set_mask(asx_layer* layer, const uint8_t* mask, int64_t rows, void* cuda_stream);
+
+/*
+ * Generate and set a mask with `rows` entries in which blocks of `block` consecutive rows
+ * (raster order, last block possibly short) are kept or dropped together.  The number of
+ * dropped blocks is floor(sparsity * nblocks + 1/2), nblocks = ceil(rows / block).  Block b
+ * gets the 64-bit score (out[1] << 32 | out[0]) of Philox4x32-10 with counter (b_lo, b_hi, 0, 0)
+ * and key (seed_lo, seed_hi); the blocks with the smallest (score, b) are dropped (a random
+ * ranking, as in Algorithm 1's getMask).  0 <= sparsity <= 1, block >= 1.
+ */
+asx_status asx_set_mask_random(asx_layer* layer, int64_t rows, double sparsity, int block,
+                               uint64_t seed, void* cuda_stream);
+
+/*
+ * Run the layer (Section 3.2 stages i-iii fused): gather the kept windows of x, multiply by
+ * the filters on the tensor cores, add the bias, apply the activation, write kept rows to
+ * their NHWC positions and zeros to the dropped ones.  Every element of y is written once.
+ *   x    : device, bf16 [Nb][H][W][C_in], 16-byte aligned when C_in % 8 == 0, else 2-byte.
+ *   w    : device, bf16 [C_out][kh][kw][C_in], same alignment rule.
+ *   bias : device, fp32 [C_out], 4-byte aligned, or NULL for zero bias.
+ *   y    : device, bf16 [Nb][Ho][Wo][C_out], Ho = (H + 2*pad - kh)/stride + 1 (Wo alike);
+ *          16-byte aligned when C_out % 8 == 0, else 2-byte; must not overlap x.
+ *   flags: OR of ASX_ACT_RELU, ASX_RECOMPACT, ASX_IMPL_NAIVE.
+ * Asynchronous on `cuda_stream`; allocates only when a layer first needs a staging buffer
+ * (C_in % 8 != 0) or when that buffer must grow.  Errors: ASX_ERR_NO_MASK, ASX_ERR_SHAPE when
+ * the mask length is neither Ho*Wo nor Nb*Ho*Wo, ASX_ERR_INVALID_ARG, ASX_ERR_ALIGN,
+ * ASX_ERR_UNSUPPORTED when Nb*Ho*Wo or a tensor's element count reaches 2^31.
+ */
+asx_status asx_run(asx_layer* layer, const void* x, int Nb, int H, int W,
+                   const void* w, const float* bias, void* y, int flags, void* cuda_stream);
+
+/*
+ * Kept-row list of the current mask.  Waits for the stream last used with this layer.
+ * *count receives the number of kept mask entries; *dev_kept a device pointer to `count`
+ * ascending int32 positions, owned by the layer and valid until the next asx_set_mask*,
+ * ASX_RECOMPACT run or asx_destroy.  Either output pointer may be NULL.
+ */
+asx_status asx_get_kept(asx_layer* layer, int64_t* count, const int32_t** dev_kept);
+
+/*
+ * Copy the kept-row list to host memory.  Waits for the stream last used with this layer.
+ * *count receives the number of kept entries; at most `capacity` of them are written to
+ * host_out (which may be NULL when capacity is 0).
+ */
+asx_status asx_get_kept_host(asx_layer* layer, int32_t* host_out, int64_t capacity, int64_t* count);
+
+/* Copy the stored mask (0/1 bytes) to host memory; `rows` must equal the stored length. */
+asx_status asx_get_mask(asx_layer* layer, uint8_t* host_mask_out, int64_t rows);
+
+/*
+ * Waits for the stream last used with this layer and reports the kernels' status word:
+ * ASX_OK, or ASX_ERR_TIMEOUT if a bounded wait inside a kernel ran out (the output of that
+ * call is then undefined; the CUDA context stays usable).  The word is cleared by the call.
+ */
+asx_status asx_last_device_status(asx_layer* layer);
+
+/* Free the layer and the device memory it owns.  NULL is allowed. */
+asx_status asx_destroy(asx_layer* layer);
+
+/*
+ * Stand-alone mask compaction (the kept-row enumeration of Algorithm 2's first function).
+ *   mask_dev  : device, `rows` bytes (0 / non-zero), any alignment.
+ *   kept_dev  : device, room for `rows` int32; receives the ascending kept positions.
+ *   count_dev : device, one int32; receives the number of kept positions.
+ *   scratch_dev, scratch_bytes : device scratch of at least asx_compact_scratch_bytes(rows)
+ *               bytes, 8-byte aligned; contents on entry are irrelevant, it is cleared on
+ *               the stream first.  Calls sharing one scratch buffer must not overlap.
+ * 0 <= rows < 2^31.  Asynchronous on `cuda_stream`; allocates nothing.
+ */
+int64_t asx_compact_scratch_bytes(int64_t rows);
+asx_status asx_compact(const uint8_t* mask_dev, int64_t rows, int32_t* kept_dev,
+                       int32_t* count_dev, void* scratch_dev, int64_t scratch_bytes,
+                       void* cuda_stream);
+/* Waits for `cuda_stream`, then reports whether the last asx_compact that used this scratch
+ * buffer ran to completion (ASX_OK) or gave up in a bounded wait (ASX_ERR_TIMEOUT). */
+asx_status asx_compact_status(const void* scratch_dev, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASX_H_ */

@@ -1,0 +1,394 @@
+// Host side of the C ABI (include/asx.h): argument checks, the layer handle and its device
+// buffers, mask generation, tensor-map encoding and the launches.  No arithmetic of the
+// method runs on the host.
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "asx_internal.h"
+
+using namespace asx;
+
+struct asx_layer {
+    int C_in, C_out, kh, kw, stride, pad;
+    int device = -1;
+    int num_sms = 0;
+    // mask state (device)
+    int64_t rows = 0, cap_rows = 0;
+    uint8_t* d_mask = nullptr;
+    int32_t* d_kept = nullptr;
+    void* d_scratch = nullptr;
+    int32_t* d_small = nullptr;        // [0] kept count, [1] status word
+    bool has_mask = false;
+    // staging for filters whose K is not a multiple of 8
+    void* d_wpack = nullptr;
+    size_t wpack_bytes = 0;
+    // tensor map cache
+    CUtensorMap tmap;
+    const void* tmap_ptr = nullptr;
+    int tmap_BN = 0, tmap_Kw = 0;
+    cudaStream_t last_stream = nullptr;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+asx_status from_cuda(cudaError_t e)
+{
+    if (e == cudaSuccess) return ASX_OK;
+    if (e == cudaErrorMemoryAllocation) return ASX_ERR_OOM;
+    return ASX_ERR_CUDA;
+}
+
+asx_status bind_device(asx_layer* L)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ASX_ERR_CUDA;
+    if (L->device < 0) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return ASX_ERR_CUDA;
+        if (prop.major != 10) return ASX_ERR_UNSUPPORTED;     // built for sm_100a only
+        L->device = dev;
+        L->num_sms = prop.multiProcessorCount;
+    } else if (L->device != dev) {
+        return ASX_ERR_INVALID_ARG;                          // a layer stays on its first device
+    }
+    return ASX_OK;
+}
+
+asx_status ensure_mask_buffers(asx_layer* L, int64_t rows)
+{
+    if (L->d_small == nullptr) {
+        if (cudaMalloc(&L->d_small, 2 * sizeof(int32_t)) != cudaSuccess) return ASX_ERR_OOM;
+        if (cudaMemset(L->d_small, 0, 2 * sizeof(int32_t)) != cudaSuccess) return ASX_ERR_CUDA;
+    }
+    if (rows <= L->cap_rows) return ASX_OK;
+    if (L->cap_rows > 0) cudaStreamSynchronize(L->last_stream);
+    cudaFree(L->d_mask); cudaFree(L->d_kept); cudaFree(L->d_scratch);
+    L->d_mask = nullptr; L->d_kept = nullptr; L->d_scratch = nullptr; L->cap_rows = 0;
+    const size_t mask_bytes = ((size_t)rows + 15) / 16 * 16;
+    if (cudaMalloc(&L->d_mask, mask_bytes) != cudaSuccess) return ASX_ERR_OOM;
+    if (cudaMalloc(&L->d_kept, sizeof(int32_t) * (size_t)rows) != cudaSuccess) return ASX_ERR_OOM;
+    if (cudaMalloc(&L->d_scratch, (size_t)compact_scratch_bytes(rows)) != cudaSuccess) return ASX_ERR_OOM;
+    L->cap_rows = rows;
+    return ASX_OK;
+}
+
+asx_status run_compaction(asx_layer* L, cudaStream_t st)
+{
+    return from_cuda(launch_compact(L->d_mask, L->rows, L->d_kept, L->d_small, L->d_scratch, st));
+}
+
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", 2011).
+void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n1 = (uint32_t)p1;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        const uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* asx_status_string(asx_status s)
+{
+    switch (s) {
+        case ASX_OK: return "ok";
+        case ASX_ERR_INVALID_ARG: return "invalid argument";
+        case ASX_ERR_UNSUPPORTED: return "unsupported configuration";
+        case ASX_ERR_NO_MASK: return "no mask set";
+        case ASX_ERR_SHAPE: return "mask length does not match the output geometry";
+        case ASX_ERR_ALIGN: return "pointer alignment";
+        case ASX_ERR_OOM: return "out of memory";
+        case ASX_ERR_CUDA: return "CUDA error";
+        case ASX_ERR_TIMEOUT: return "bounded wait in a kernel ran out";
+    }
+    return "unknown status";
+}
+
+asx_status asx_create_layer(int C_in, int C_out, int kh, int kw, int stride, int pad, asx_layer** out)
+{
+    if (out == nullptr) return ASX_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (C_in < 1 || C_out < 1 || kh < 1 || kw < 1 || stride < 1 || pad < 0) return ASX_ERR_INVALID_ARG;
+    if ((int64_t)kh * kw * C_in >= (1ll << 24) || C_out >= (1 << 20) || kh > 255 || kw > 255 || pad > 255)
+        return ASX_ERR_UNSUPPORTED;
+    asx_layer* L = new (std::nothrow) asx_layer();
+    if (L == nullptr) return ASX_ERR_OOM;
+    L->C_in = C_in; L->C_out = C_out; L->kh = kh; L->kw = kw; L->stride = stride; L->pad = pad;
+    *out = L;
+    return ASX_OK;
+}
+
+asx_status asx_set_mask(asx_layer* L, const uint8_t* mask, int64_t rows, void* cuda_stream)
+{
+    if (L == nullptr || mask == nullptr) return ASX_ERR_INVALID_ARG;
+    if (rows < 1 || rows >= (1ll << 31)) return ASX_ERR_INVALID_ARG;
+    asx_status s = bind_device(L);
+    if (s != ASX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    s = ensure_mask_buffers(L, rows);
+    if (s != ASX_OK) return s;
+    cudaPointerAttributes attr;
+    bool on_device = false;
+    if (cudaPointerGetAttributes(&attr, mask) == cudaSuccess)
+        on_device = (attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged);
+    else
+        cudaGetLastError();
+    cudaError_t e;
+    if (on_device) {
+        e = cudaMemcpyAsync(L->d_mask, mask, (size_t)rows, cudaMemcpyDeviceToDevice, st);
+    } else {
+        e = cudaMemcpyAsync(L->d_mask, mask, (size_t)rows, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);      // the caller may free a host mask on return
+    }
+    if (e != cudaSuccess) return from_cuda(e);
+    L->rows = rows;
+    L->last_stream = st;
+    s = run_compaction(L, st);
+    L->has_mask = (s == ASX_OK);
+    return s;
+}
+
+asx_status asx_set_mask_random(asx_layer* L, int64_t rows, double sparsity, int block, uint64_t seed,
+                               void* cuda_stream)
+{
+    if (L == nullptr) return ASX_ERR_INVALID_ARG;
+    if (rows < 1 || rows >= (1ll << 31) || block < 1 || !(sparsity >= 0.0 && sparsity <= 1.0))
+        return ASX_ERR_INVALID_ARG;
+    const int64_t nblocks = (rows + block - 1) / block;
+    int64_t n_drop = (int64_t)(sparsity * (double)nblocks + 0.5);
+    if (n_drop > nblocks) n_drop = nblocks;
+    std::vector<uint8_t> mask;
+    std::vector<std::pair<uint64_t, int64_t>> score;
+    try {
+        mask.assign((size_t)rows, 1);
+        score.resize((size_t)nblocks);
+    } catch (const std::bad_alloc&) {
+        return ASX_ERR_OOM;
+    }
+    const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    for (int64_t b = 0; b < nblocks; ++b) {
+        const uint32_t ctr[4] = {(uint32_t)b, (uint32_t)((uint64_t)b >> 32), 0u, 0u};
+        uint32_t o[4];
+        philox4x32_10(ctr, key, o);
+        score[(size_t)b] = {((uint64_t)o[1] << 32) | o[0], b};
+    }
+    if (n_drop > 0 && n_drop < nblocks)
+        std::nth_element(score.begin(), score.begin() + (n_drop - 1), score.end());
+    for (int64_t i = 0; i < n_drop; ++i) {
+        const int64_t b = score[(size_t)i].second;
+        const int64_t lo = b * block, hi = std::min<int64_t>(rows, lo + block);
+        std::memset(mask.data() + lo, 0, (size_t)(hi - lo));
+    }
+    return asx_set_mask(L, mask.data(), rows, cuda_stream);
+}
+
+asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void* w, const float* bias,
+                   void* y, int flags, void* cuda_stream)
+{
+    if (L == nullptr || x == nullptr || w == nullptr || y == nullptr) return ASX_ERR_INVALID_ARG;
+    if (Nb < 1 || H < 1 || W < 1) return ASX_ERR_INVALID_ARG;
+    if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE)) return ASX_ERR_INVALID_ARG;
+    if (H + 2 * L->pad < L->kh || W + 2 * L->pad < L->kw) return ASX_ERR_INVALID_ARG;
+    if (!L->has_mask) return ASX_ERR_NO_MASK;
+    asx_status s = bind_device(L);
+    if (s != ASX_OK) return s;
+
+    ConvGeom g;
+    g.Nb = Nb; g.H = H; g.W = W; g.C_in = L->C_in; g.C_out = L->C_out;
+    g.kh = L->kh; g.kw = L->kw; g.stride = L->stride; g.pad = L->pad;
+    g.Ho = (H + 2 * L->pad - L->kh) / L->stride + 1;
+    g.Wo = (W + 2 * L->pad - L->kw) / L->stride + 1;
+    g.K = L->kh * L->kw * L->C_in;
+    const int64_t P = (int64_t)g.Ho * g.Wo, M = P * Nb;
+    const int64_t lim = (1ll << 31) - 1;
+    if (H > 32767 || W > 32767) return ASX_ERR_UNSUPPORTED;
+    if (M > lim || (int64_t)Nb * H * W * L->C_in > lim || M * L->C_out > lim) return ASX_ERR_UNSUPPORTED;
+    if (L->rows != P && L->rows != M) return ASX_ERR_SHAPE;
+    g.P = (int)P; g.M = (int)M; g.rows = (int)L->rows;
+
+    const bool vec_in = (L->C_in % 8 == 0);
+    const uintptr_t in_align = vec_in ? 15 : 1;
+    if ((reinterpret_cast<uintptr_t>(x) & in_align) || (reinterpret_cast<uintptr_t>(w) & in_align))
+        return ASX_ERR_ALIGN;
+    if (reinterpret_cast<uintptr_t>(y) & ((L->C_out % 8 == 0) ? 15 : 1)) return ASX_ERR_ALIGN;
+    if (bias != nullptr && (reinterpret_cast<uintptr_t>(bias) & 3)) return ASX_ERR_ALIGN;
+    {
+        const uintptr_t xb = reinterpret_cast<uintptr_t>(x), xe = xb + (uintptr_t)Nb * H * W * L->C_in * 2;
+        const uintptr_t yb = reinterpret_cast<uintptr_t>(y), ye = yb + (uintptr_t)M * L->C_out * 2;
+        if (xb < ye && yb < xe) return ASX_ERR_INVALID_ARG;
+    }
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    L->last_stream = st;
+    if (flags & ASX_RECOMPACT) {
+        s = run_compaction(L, st);
+        if (s != ASX_OK) return s;
+    }
+    const int relu = (flags & ASX_ACT_RELU) ? 1 : 0;
+    int32_t* d_count = L->d_small;
+    int* d_status = reinterpret_cast<int*>(L->d_small + 1);
+
+    if (flags & ASX_IMPL_NAIVE)
+        return from_cuda(launch_naive(g, x, w, bias, y, L->d_mask, L->d_kept, d_count, relu, st));
+
+    FastPlan plan;
+    if (!plan_fast(g, &plan)) return ASX_ERR_UNSUPPORTED;
+    const void* wsrc = w;
+    int Kw = g.K;
+    if (!plan.vec) {
+        // filters whose rows are not a multiple of 16 bytes are staged into a padded copy
+        Kw = (g.K + 7) / 8 * 8;
+        const size_t need = (size_t)L->C_out * Kw * 2;
+        if (need > L->wpack_bytes) {
+            cudaStreamSynchronize(st);
+            cudaFree(L->d_wpack);
+            L->d_wpack = nullptr; L->wpack_bytes = 0;
+            if (cudaMalloc(&L->d_wpack, need) != cudaSuccess) return ASX_ERR_OOM;
+            L->wpack_bytes = need;
+            L->tmap_ptr = nullptr;
+        }
+        cudaError_t e = launch_repack_w(w, L->d_wpack, L->C_out, g.K, Kw, st);
+        if (e != cudaSuccess) return from_cuda(e);
+        wsrc = L->d_wpack;
+    }
+    if (L->tmap_ptr != wsrc || L->tmap_BN != plan.BN || L->tmap_Kw != Kw) {
+        EncodeTiledFn enc = encode_tiled_fn();
+        if (enc == nullptr) return ASX_ERR_CUDA;
+        const cuuint64_t dims[2] = {(cuuint64_t)Kw, (cuuint64_t)L->C_out};
+        const cuuint64_t strides[1] = {(cuuint64_t)Kw * 2};
+        const cuuint32_t box[2] = {64u, (cuuint32_t)plan.BN};
+        const cuuint32_t estr[2] = {1u, 1u};
+        const CUresult r = enc(&L->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(wsrc), dims,
+                               strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return ASX_ERR_CUDA;
+        L->tmap_ptr = wsrc; L->tmap_BN = plan.BN; L->tmap_Kw = Kw;
+    }
+    return from_cuda(launch_fast(g, plan, L->tmap, x, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
+                                 L->num_sms, st));
+}
+
+asx_status asx_get_kept(asx_layer* L, int64_t* count, const int32_t** dev_kept)
+{
+    if (L == nullptr) return ASX_ERR_INVALID_ARG;
+    if (!L->has_mask) return ASX_ERR_NO_MASK;
+    if (cudaStreamSynchronize(L->last_stream) != cudaSuccess) return ASX_ERR_CUDA;
+    int32_t c = 0;
+    if (cudaMemcpy(&c, L->d_small, sizeof(c), cudaMemcpyDeviceToHost) != cudaSuccess) return ASX_ERR_CUDA;
+    if (count) *count = c;
+    if (dev_kept) *dev_kept = L->d_kept;
+    return ASX_OK;
+}
+
+asx_status asx_get_kept_host(asx_layer* L, int32_t* host_out, int64_t capacity, int64_t* count)
+{
+    if (L == nullptr || count == nullptr || capacity < 0 || (capacity > 0 && host_out == nullptr))
+        return ASX_ERR_INVALID_ARG;
+    int64_t c = 0;
+    const asx_status s = asx_get_kept(L, &c, nullptr);
+    if (s != ASX_OK) return s;
+    *count = c;
+    const int64_t n = c < capacity ? c : capacity;
+    if (n > 0 && cudaMemcpy(host_out, L->d_kept, sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return ASX_ERR_CUDA;
+    return ASX_OK;
+}
+
+asx_status asx_get_mask(asx_layer* L, uint8_t* host_mask_out, int64_t rows)
+{
+    if (L == nullptr || host_mask_out == nullptr) return ASX_ERR_INVALID_ARG;
+    if (!L->has_mask) return ASX_ERR_NO_MASK;
+    if (rows != L->rows) return ASX_ERR_SHAPE;
+    if (cudaStreamSynchronize(L->last_stream) != cudaSuccess) return ASX_ERR_CUDA;
+    return from_cuda(cudaMemcpy(host_mask_out, L->d_mask, (size_t)rows, cudaMemcpyDeviceToHost));
+}
+
+asx_status asx_last_device_status(asx_layer* L)
+{
+    if (L == nullptr) return ASX_ERR_INVALID_ARG;
+    if (L->d_small == nullptr) return ASX_OK;
+    if (cudaStreamSynchronize(L->last_stream) != cudaSuccess) return ASX_ERR_CUDA;
+    int32_t word = 0;
+    if (cudaMemcpy(&word, L->d_small + 1, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return ASX_ERR_CUDA;
+    int32_t scan_err = 0;
+    if (L->d_scratch != nullptr &&
+        cudaMemcpy(&scan_err, static_cast<int32_t*>(L->d_scratch) + 1, sizeof(scan_err), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return ASX_ERR_CUDA;
+    if (word != 0 && cudaMemset(L->d_small + 1, 0, sizeof(word)) != cudaSuccess) return ASX_ERR_CUDA;
+    return (word != 0 || scan_err != 0) ? ASX_ERR_TIMEOUT : ASX_OK;
+}
+
+asx_status asx_destroy(asx_layer* L)
+{
+    if (L == nullptr) return ASX_OK;
+    if (L->device >= 0) {
+        cudaStreamSynchronize(L->last_stream);
+        cudaFree(L->d_mask); cudaFree(L->d_kept); cudaFree(L->d_scratch);
+        cudaFree(L->d_small); cudaFree(L->d_wpack);
+    }
+    delete L;
+    return ASX_OK;
+}
+
+int64_t asx_compact_scratch_bytes(int64_t rows)
+{
+    if (rows < 0) return 0;
+    return compact_scratch_bytes(rows);
+}
+
+asx_status asx_compact(const uint8_t* mask_dev, int64_t rows, int32_t* kept_dev, int32_t* count_dev,
+                       void* scratch_dev, int64_t scratch_bytes, void* cuda_stream)
+{
+    if (rows < 0 || rows >= (1ll << 31) || count_dev == nullptr || scratch_dev == nullptr) return ASX_ERR_INVALID_ARG;
+    if (rows > 0 && (mask_dev == nullptr || kept_dev == nullptr)) return ASX_ERR_INVALID_ARG;
+    if (scratch_bytes < compact_scratch_bytes(rows)) return ASX_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(scratch_dev) & 7) return ASX_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(kept_dev) & 3) || (reinterpret_cast<uintptr_t>(count_dev) & 3)) return ASX_ERR_ALIGN;
+    return from_cuda(launch_compact(mask_dev, rows, kept_dev, count_dev, scratch_dev,
+                                    static_cast<cudaStream_t>(cuda_stream)));
+}
+
+asx_status asx_compact_status(const void* scratch_dev, void* cuda_stream)
+{
+    if (scratch_dev == nullptr) return ASX_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return ASX_ERR_CUDA;
+    int32_t err = 0;
+    if (cudaMemcpy(&err, static_cast<const int32_t*>(scratch_dev) + 1, sizeof(err), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return ASX_ERR_CUDA;
+    return err != 0 ? ASX_ERR_TIMEOUT : ASX_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,164 @@
+// S1 — mask compaction: kept[j] = position of the j-th non-zero mask byte, ascending.
+//
+// Appendix A, Algorithm 2 (first function) walks the output positions in raster order and
+// appends an entry for every position whose mask is 1; the running index of that loop is an
+// exclusive prefix sum of the mask.  Here the prefix sum is a single-pass chained scan:
+// each 4096-row tile counts its kept rows (16 mask bytes per thread, popcount, a shuffle
+// scan inside each warp and across the warp totals), publishes its total, and finds the
+// number of kept rows before it by looking back over its predecessors' published values,
+// 32 predecessors at a time with a warp ballot.  Tiles take their numbers from an atomic
+// ticket so that every predecessor of a running tile has already started; the look-back
+// wait is bounded and reports through the error word instead of spinning for ever.
+#include "asx_internal.h"
+
+namespace asx {
+
+namespace {
+
+constexpr unsigned long long FLAG_AGGREGATE = 1ull << 32;   // value = this tile's own count
+constexpr unsigned long long FLAG_INCLUSIVE = 2ull << 32;   // value = count up to and including this tile
+constexpr long long LOOKBACK_CYCLE_LIMIT = 2000000000ll;    // about one second
+
+struct ScratchHeader {
+    unsigned int ticket;
+    int error;
+};
+
+__device__ __forceinline__ unsigned nonzero_bytes4(unsigned w)
+{
+    unsigned t = ((w & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w;     // bit 7 of each byte: byte != 0
+    return ((t >> 7) & 1u) | ((t >> 14) & 2u) | ((t >> 21) & 4u) | ((t >> 28) & 8u);
+}
+
+__global__ void __launch_bounds__(COMPACT_THREADS)
+compact_kernel(const uint8_t* __restrict__ mask, long long rows, int32_t* __restrict__ kept,
+               int32_t* __restrict__ count, ScratchHeader* hdr,
+               volatile unsigned long long* status, int num_tiles)
+{
+    __shared__ int32_t s_idx[COMPACT_TILE];
+    __shared__ int s_warp_total[COMPACT_THREADS / 32];
+    __shared__ int s_tile;
+    __shared__ int s_exclusive;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) s_tile = (int)atomicAdd(&hdr->ticket, 1u);
+    __syncthreads();
+    const int tile = s_tile;
+    if (tile >= num_tiles) return;
+
+    // 16 mask bytes per thread -> 16 flag bits
+    const long long first = (long long)tile * COMPACT_TILE + (long long)tid * COMPACT_PER_THREAD;
+    unsigned flags = 0;
+    const bool aligned = (reinterpret_cast<uintptr_t>(mask) & 15) == 0;
+    if (aligned && first + COMPACT_PER_THREAD <= rows) {
+        const uint4 v = *reinterpret_cast<const uint4*>(mask + first);
+        flags = nonzero_bytes4(v.x) | (nonzero_bytes4(v.y) << 4) | (nonzero_bytes4(v.z) << 8) |
+                (nonzero_bytes4(v.w) << 12);
+    } else {
+        for (int j = 0; j < COMPACT_PER_THREAD; ++j)
+            if (first + j < rows && mask[first + j] != 0) flags |= 1u << j;
+    }
+    const int mine = __popc(flags);
+
+    // inclusive shuffle scan inside the warp, then over the warp totals
+    int incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += t;
+    }
+    if (lane == 31) s_warp_total[warp] = incl;
+    __syncthreads();
+    int warp_prefix = 0, tile_total = 0;
+#pragma unroll
+    for (int i = 0; i < COMPACT_THREADS / 32; ++i) {
+        const int t = s_warp_total[i];
+        if (i < warp) warp_prefix += t;
+        tile_total += t;
+    }
+
+    // chained scan across tiles
+    if (warp == 0) {
+        if (tile == 0) {
+            if (lane == 0) {
+                status[0] = FLAG_INCLUSIVE | (unsigned)tile_total;
+                s_exclusive = 0;
+            }
+        } else {
+            if (lane == 0) status[tile] = FLAG_AGGREGATE | (unsigned)tile_total;
+            int exclusive = 0;
+            int idx = tile - 1 - lane;
+            bool failed = false;
+            while (true) {
+                unsigned long long st = FLAG_INCLUSIVE;       // before tile 0: nothing kept
+                if (idx >= 0) {
+                    st = status[idx];
+                    if ((st >> 32) == 0) {
+                        const long long t0 = clock64();
+                        while (((st = status[idx]) >> 32) == 0) {
+                            if (clock64() - t0 > LOOKBACK_CYCLE_LIMIT) { failed = true; break; }
+                            __nanosleep(40);
+                        }
+                    }
+                }
+                if (__any_sync(0xffffffffu, failed)) { failed = true; break; }
+                const unsigned has_inclusive = __ballot_sync(0xffffffffu, (st >> 32) == 2);
+                const int stop = __ffs(has_inclusive) - 1;    // nearest predecessor with a full prefix
+                int v = (stop < 0 || lane <= stop) ? (int)(unsigned)(st & 0xffffffffu) : 0;
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+                exclusive += v;
+                if (stop >= 0) break;
+                idx -= 32;
+            }
+            if (lane == 0) {
+                if (failed) {
+                    atomicOr(&hdr->error, DEV_TIMEOUT_SCAN);
+                    exclusive = 0;
+                }
+                status[tile] = FLAG_INCLUSIVE | (unsigned)(exclusive + tile_total);
+                s_exclusive = exclusive;
+            }
+        }
+    }
+
+    // ordered write: into shared memory first, then coalesced to the list
+    int at = warp_prefix + incl - mine;
+    unsigned f = flags;
+    while (f) {
+        const int j = __ffs(f) - 1;
+        f &= f - 1;
+        s_idx[at++] = (int32_t)(first + j);
+    }
+    __syncthreads();
+    const int exclusive = s_exclusive;
+    for (int i = tid; i < tile_total; i += COMPACT_THREADS) kept[exclusive + i] = s_idx[i];
+    if (tile == num_tiles - 1 && tid == 0) *count = exclusive + tile_total;
+}
+
+}  // namespace
+
+static int tiles_for(int64_t rows)
+{
+    int64_t t = (rows + COMPACT_TILE - 1) / COMPACT_TILE;
+    return (int)(t < 1 ? 1 : t);
+}
+
+int64_t compact_scratch_bytes(int64_t rows)
+{
+    return (int64_t)sizeof(ScratchHeader) + 8 * (int64_t)tiles_for(rows);
+}
+
+cudaError_t launch_compact(const uint8_t* mask, int64_t rows, int32_t* kept, int32_t* count,
+                           void* scratch, cudaStream_t st)
+{
+    const int tiles = tiles_for(rows);
+    cudaError_t e = cudaMemsetAsync(scratch, 0, (size_t)compact_scratch_bytes(rows), st);
+    if (e != cudaSuccess) return e;
+    auto* hdr = static_cast<ScratchHeader*>(scratch);
+    auto* status = reinterpret_cast<unsigned long long*>(hdr + 1);
+    compact_kernel<<<tiles, COMPACT_THREADS, 0, st>>>(mask, (long long)rows, kept, count, hdr, status, tiles);
+    return cudaGetLastError();
+}
+
+}  // namespace asx

@@ -1,0 +1,468 @@
+// S2 + S3 + S4 — the masked convolution as one persistent, warp-specialised sm_100a kernel.
+//
+// Section 3.2 / Appendix A describe three stages: an indirection-based lowering that skips
+// masked positions, an unmodified dense GEMM over the reduced range, and a post-processing
+// pass that re-inserts zeros.  Here the three are one kernel over tiles of 128 kept rows:
+//
+//   producer warps  gather the kept windows of x straight into the shared-memory operand
+//                   layout the tensor core reads (K-major rows of 64 bf16 with the 128-byte
+//                   swizzle); nothing is lowered to global memory.  Padding taps and rows
+//                   past the end of the kept list are filled with zeros.
+//   TMA thread      streams the matching 64-wide K slab of the filter matrix w[C_out][K].
+//   MMA thread      issues tcgen05.mma (128 x BN x 16, bf16 -> fp32) into one of two
+//                   accumulators in tensor memory, so the epilogue of tile i overlaps the
+//                   main loop of tile i+1.
+//   epilogue warps  first write zeros to the dropped output rows that lie between this
+//                   tile's first kept row and the next tile's first kept row (kept rows are
+//                   ascending, so these intervals partition the output), then read the
+//                   accumulator, add the bias, apply ReLU, round to bf16 and store each kept
+//                   row at its NHWC position.  Every output element is written exactly once.
+//
+// The kept-row count is read from device memory, so the host never has to know it.
+// All waits are bounded: a wait that runs out sets the status word and every role leaves.
+#include <cuda_bf16.h>
+#include "asx_internal.h"
+#include "ptx_sm100.cuh"
+
+namespace asx {
+
+namespace {
+
+constexpr int BM = 128;                 // kept rows per tile (UMMA M)
+constexpr int BK = 64;                  // K elements per pipeline stage (one 128-byte swizzled row)
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int MAX_STAGES = 8;
+constexpr int LAG = 2;                  // cp.async groups a producer thread keeps in flight
+constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_EPI0 = 2, WARP_PROD0 = 6;
+constexpr int NUM_PROD_WARPS = 4, NUM_EPI_WARPS = 4;
+constexpr int NUM_THREADS = 32 * (WARP_PROD0 + NUM_PROD_WARPS);
+constexpr long long WAIT_CYCLE_LIMIT = 4000000000ll;   // about two seconds
+
+struct FastArgs {
+    const __nv_bfloat16* x;
+    const float* bias;
+    __nv_bfloat16* y;
+    const uint8_t* mask;
+    const int32_t* kept;
+    const int32_t* count;
+    int* dev_status;
+    int relu;
+    int BN, n_tiles, stages, tmem_cols;
+    int vec_out;        // C_out % 8 == 0 and y 16-byte aligned: 16-byte stores
+};
+
+struct Shared {           // lives after the operand stages
+    unsigned long long full[MAX_STAGES];
+    unsigned long long empty[MAX_STAGES];
+    unsigned long long acc_full[2];
+    unsigned long long acc_empty[2];
+    unsigned int tmem_base;
+    int abort;
+};
+
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                         int* dev_status)
+{
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > WAIT_CYCLE_LIMIT) {
+            *abort_flag = 1;
+            atomicOr(dev_status, DEV_TIMEOUT_PIPE);
+            return false;
+        }
+    }
+    return true;
+}
+
+// Output row (n*P + p) of the rk-th kept lowered row.
+__device__ __forceinline__ int out_row_of(int rk, int cnt, const ConvGeom& g, const int32_t* __restrict__ kept)
+{
+    if (g.rows == g.P) {
+        const int n = rk / cnt;
+        return n * g.P + __ldg(kept + (rk - n * cnt));
+    }
+    return __ldg(kept + rk);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvGeom g, const FastArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    const int cnt = *a.count;
+    const int Mk = (g.rows == g.P) ? g.Nb * cnt : cnt;
+    const int N = g.C_out;
+
+    if (Mk <= 0) {
+        // every position dropped: the whole output is zeros (Algorithm 2, mask == 0 branch)
+        const long long total = (long long)g.M * N;
+        const long long t = blockIdx.x * (long long)NUM_THREADS + tid, step = (long long)gridDim.x * NUM_THREADS;
+        if (a.vec_out) {
+            uint4* y16 = reinterpret_cast<uint4*>(a.y);
+            for (long long i = t; i < total / 8; i += step) y16[i] = make_uint4(0, 0, 0, 0);
+        } else {
+            unsigned short* y2 = reinterpret_cast<unsigned short*>(a.y);
+            for (long long i = t; i < total; i += step) y2[i] = 0;
+        }
+        return;
+    }
+
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int BN = a.BN, S = a.stages;
+    const int stage_bytes = A_STAGE_BYTES + BN * (BK * 2);
+    Shared* sh = reinterpret_cast<Shared*>(smem_raw + (smem_base - ptx::smem_u32(smem_raw)) + S * stage_bytes);
+    volatile int* abort_flag = &sh->abort;
+
+    const int KB = (g.K + BK - 1) / BK;
+    const int m_tiles = (Mk + BM - 1) / BM;
+    const int total_tiles = m_tiles * a.n_tiles;
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1 + NUM_PROD_WARPS);
+            ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&sh->acc_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh->acc_empty[i]), NUM_EPI_WARPS);
+        }
+        sh->abort = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == WARP_MMA) {
+        ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), (uint32_t)a.tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    if (warp == WARP_TMA && lane == 0) ptx::prefetch_tensormap(&tmap_w);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = sh->tmem_base;
+
+    if (warp == WARP_TMA) {
+        // ------------------------------------------------------------------ filter slabs by TMA
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const int n_tile = t % a.n_tiles;
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = it % S;
+                    const uint32_t ph = (uint32_t)(it / S) & 1u;
+                    if (!wait_bar(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
+                    const uint32_t full = ptx::smem_u32(&sh->full[s]);
+                    ptx::mbar_arrive_expect_tx(full, (uint32_t)(BN * BK * 2));
+                    ptx::tma_load_2d(smem_base + s * stage_bytes + A_STAGE_BYTES, &tmap_w, full, kb * BK, n_tile * BN);
+                }
+            }
+            if (!ok) {   // let loads already issued land before the block's shared memory goes away
+                for (int i = 0; i < 64; ++i) __nanosleep(1000);
+            }
+        }
+    } else if (warp == WARP_MMA) {
+        // ------------------------------------------------------------------ MMA issue
+        if (lane == 0) {
+            const uint32_t idesc = ptx::umma_idesc_bf16(BM, BN);
+            int it = 0, ti = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
+                const int buf = ti & 1;
+                const uint32_t use = (uint32_t)(ti >> 1) & 1u;
+                if (!wait_bar(ptx::smem_u32(&sh->acc_empty[buf]), use ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
+                ptx::tc_fence_after_sync();
+                const uint32_t d = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = it % S;
+                    const uint32_t ph = (uint32_t)(it / S) & 1u;
+                    if (!wait_bar(ptx::smem_u32(&sh->full[s]), ph, abort_flag, a.dev_status)) { ok = false; break; }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_addr = smem_base + s * stage_bytes;
+                    const uint64_t adesc = ptx::umma_desc_k_major_sw128(a_addr);
+                    const uint64_t bdesc = ptx::umma_desc_k_major_sw128(a_addr + A_STAGE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)      // 16 K-elements = 32 bytes = 2 descriptor units
+                        ptx::umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    ptx::umma_commit(ptx::smem_u32(&sh->empty[s]));
+                }
+                if (ok) ptx::umma_commit(ptx::smem_u32(&sh->acc_full[buf]));
+            }
+        }
+    } else if (warp < WARP_PROD0) {
+        // ------------------------------------------------------------------ epilogue
+        const int q = warp & 3;                       // TMEM lanes 32q .. 32q+31 belong to this warp
+        const int et = (warp - WARP_EPI0) * 32 + lane;
+        unsigned short* y2 = reinterpret_cast<unsigned short*>(a.y);
+        int ti = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
+            const int m_tile = t / a.n_tiles, n_tile = t - m_tile * a.n_tiles;
+            const int n0 = n_tile * BN;
+            const int ncols = min(N - n0, BN);
+            // zeros for the dropped rows this tile owns
+            {
+                const int lo = (m_tile == 0) ? 0 : out_row_of(m_tile * BM, cnt, g, a.kept);
+                const int hi = (m_tile == m_tiles - 1) ? g.M : out_row_of((m_tile + 1) * BM, cnt, g, a.kept);
+                if (a.vec_out) {
+                    const int cpr = ncols >> 3;
+                    const long long total = (long long)(hi - lo) * cpr;
+                    for (long long i = et; i < total; i += NUM_EPI_WARPS * 32) {
+                        const int rr = (int)(i / cpr), cc = (int)(i - (long long)rr * cpr);
+                        const int row = lo + rr;
+                        const int p = (g.rows == g.P) ? row % g.P : row;
+                        if (__ldg(a.mask + p) == 0)
+                            *reinterpret_cast<uint4*>(y2 + (long long)row * N + n0 + cc * 8) = make_uint4(0, 0, 0, 0);
+                    }
+                } else {
+                    const long long total = (long long)(hi - lo) * ncols;
+                    for (long long i = et; i < total; i += NUM_EPI_WARPS * 32) {
+                        const int rr = (int)(i / ncols), cc = (int)(i - (long long)rr * ncols);
+                        const int row = lo + rr;
+                        const int p = (g.rows == g.P) ? row % g.P : row;
+                        if (__ldg(a.mask + p) == 0) y2[(long long)row * N + n0 + cc] = 0;
+                    }
+                }
+            }
+            // kept rows from the accumulator
+            const int buf = ti & 1;
+            const uint32_t use = (uint32_t)(ti >> 1) & 1u;
+            const int rk = m_tile * BM + q * 32 + lane;
+            const bool valid = rk < Mk;
+            const long long yoff = valid ? (long long)out_row_of(rk, cnt, g, a.kept) * N : 0;
+            if (!wait_bar(ptx::smem_u32(&sh->acc_full[buf]), use, abort_flag, a.dev_status)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                const int col0 = n0 + c0;
+                if (col0 >= N) break;
+                uint32_t r[16];
+                ptx::tmem_ld_16(tacc + (uint32_t)c0, r);
+                ptx::tmem_ld_wait();
+                if (valid) {
+                    float v[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int col = col0 + j;
+                        float f = __uint_as_float(r[j]);
+                        if (a.bias != nullptr && col < N) f += __ldg(a.bias + col);
+                        v[j] = a.relu ? fmaxf(f, 0.f) : f;
+                    }
+                    if (a.vec_out) {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if (col0 + 8 * h < N) {
+                                uint4 o;
+                                o.x = pack_bf16(v[8 * h + 0], v[8 * h + 1]);
+                                o.y = pack_bf16(v[8 * h + 2], v[8 * h + 3]);
+                                o.z = pack_bf16(v[8 * h + 4], v[8 * h + 5]);
+                                o.w = pack_bf16(v[8 * h + 6], v[8 * h + 7]);
+                                *reinterpret_cast<uint4*>(y2 + yoff + col0 + 8 * h) = o;
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (col0 + j < N)
+                                y2[yoff + col0 + j] = __bfloat16_as_ushort(__float2bfloat16_rn(v[j]));
+                    }
+                }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[buf]));
+        }
+    } else {
+        // ------------------------------------------------------------------ gather producers
+        const int pw = warp - WARP_PROD0;
+        const int c = lane & 7;                        // 16-byte chunk of the 128-byte row
+        const int rsub = pw * 4 + (lane >> 3);         // row within each group of 16
+        const uint32_t sw_off = (uint32_t)(rsub * 128 + ((c ^ (rsub & 7)) << 4));
+        const unsigned short* x2 = reinterpret_cast<const unsigned short*>(a.x);
+        int it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const int m_tile = t / a.n_tiles;
+            int pix[8], iy0[8], ix0[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int rk = m_tile * BM + i * 16 + rsub;
+                pix[i] = 0; ix0[i] = 0; iy0[i] = -(1 << 24);          // no tap is in bounds
+                if (rk < Mk) {
+                    const int row = out_row_of(rk, cnt, g, a.kept);
+                    if ((unsigned)row < (unsigned)g.M) {
+                        const int n = row / g.P, p = row - n * g.P;
+                        const int oy = p / g.Wo, ox = p - oy * g.Wo;
+                        iy0[i] = oy * g.stride - g.pad;
+                        ix0[i] = ox * g.stride - g.pad;
+                        pix[i] = (n * g.H + iy0[i]) * g.W + ix0[i];
+                    } else {
+                        atomicOr(a.dev_status, DEV_BAD_INDEX);
+                    }
+                }
+            }
+            for (int kb = 0; kb < KB; ++kb, ++it) {
+                const int s = it % S;
+                const uint32_t ph = (uint32_t)(it / S) & 1u;
+                if (!wait_bar(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
+                const uint32_t dst0 = smem_base + s * stage_bytes + sw_off;
+                if (VEC) {
+                    const int k = kb * BK + c * 8;
+                    const bool kvalid = k < g.K;
+                    const int tap = k / g.C_in, ci = k - tap * g.C_in;
+                    const int ky = tap / g.kw, kx = tap - ky * g.kw;
+                    const int koff = ky * g.W + kx;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const bool in = kvalid && (unsigned)(iy0[i] + ky) < (unsigned)g.H &&
+                                        (unsigned)(ix0[i] + kx) < (unsigned)g.W;
+                        const unsigned short* src = in ? x2 + ((long long)(pix[i] + koff) * g.C_in + ci) : x2;
+                        ptx::cp_async_16(dst0 + i * (16 * 128), src, in ? 16u : 0u);
+                    }
+                    ptx::cp_async_commit();
+                    if (it >= LAG) {
+                        ptx::cp_async_wait<LAG>();
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->full[(it - LAG) % S]));
+                    }
+                } else {
+                    int eoff[8], eky[8], ekx[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int k = kb * BK + c * 8 + e;
+                        const int tap = k / g.C_in, ci = k - tap * g.C_in;
+                        const int ky = tap / g.kw;
+                        eky[e] = (k < g.K) ? ky : (1 << 26);                  // past K: never in bounds
+                        ekx[e] = tap - ky * g.kw;
+                        eoff[e] = (ky * g.W + ekx[e]) * g.C_in + ci;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        unsigned short e16[8];
+                        const long long base = (long long)pix[i] * g.C_in;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const bool in = (unsigned)(iy0[i] + eky[e]) < (unsigned)g.H &&
+                                            (unsigned)(ix0[i] + ekx[e]) < (unsigned)g.W;
+                            e16[e] = in ? __ldg(x2 + base + eoff[e]) : (unsigned short)0;
+                        }
+                        uint4 v;
+                        v.x = e16[0] | ((uint32_t)e16[1] << 16);
+                        v.y = e16[2] | ((uint32_t)e16[3] << 16);
+                        v.z = e16[4] | ((uint32_t)e16[5] << 16);
+                        v.w = e16[6] | ((uint32_t)e16[7] << 16);
+                        ptx::st_shared_v4(dst0 + i * (16 * 128), v);
+                    }
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->full[s]));
+                }
+            }
+        }
+        if (VEC) {
+            ptx::cp_async_wait<0>();
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (ok && lane == 0) {
+                for (int j = (it > LAG ? it - LAG : 0); j < it; ++j)
+                    ptx::mbar_arrive(ptx::smem_u32(&sh->full[j % S]));
+            }
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == WARP_MMA) {
+        __syncwarp();
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
+    }
+}
+
+__global__ void repack_w_kernel(const unsigned short* __restrict__ w, unsigned short* __restrict__ wp,
+                                int C_out, int K, int Kw)
+{
+    const long long total = (long long)C_out * Kw;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const int co = (int)(i / Kw), k = (int)(i - (long long)co * Kw);
+        wp[i] = (k < K) ? w[(long long)co * K + k] : (unsigned short)0;
+    }
+}
+
+}  // namespace
+
+bool plan_fast(const ConvGeom& g, FastPlan* plan)
+{
+    const int N = g.C_out;
+    const int n_tiles = (N + 255) / 256;
+    const int per = (N + n_tiles - 1) / n_tiles;
+    const int BN = ((per + 15) / 16) * 16;
+    const int stage_bytes = A_STAGE_BYTES + BN * BK * 2;
+    const int budget = 227 * 1024 - 1024 - (int)sizeof(Shared);
+    int S = budget / stage_bytes;
+    if (S > MAX_STAGES) S = MAX_STAGES;
+    if (S < LAG + 2) return false;
+    plan->BN = BN;
+    plan->n_tiles = n_tiles;
+    plan->stages = S;
+    int smem = 1024 + S * stage_bytes + (int)sizeof(Shared);
+    if (smem < 120 * 1024) smem = 120 * 1024;      // one block per SM: tensor memory is not shared out
+    plan->smem_bytes = smem;
+    plan->vec = (g.C_in % 8 == 0) ? 1 : 0;
+    plan->Kpad = ((g.K + BK - 1) / BK) * BK;
+    return true;
+}
+
+cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorMap& tmap_w,
+                        const void* x, const float* bias, void* y, const uint8_t* mask,
+                        const int32_t* kept, const int32_t* count, int relu, int* dev_status,
+                        int num_sms, cudaStream_t st)
+{
+    FastArgs a;
+    a.x = static_cast<const __nv_bfloat16*>(x);
+    a.bias = bias;
+    a.y = static_cast<__nv_bfloat16*>(y);
+    a.mask = mask;
+    a.kept = kept;
+    a.count = count;
+    a.dev_status = dev_status;
+    a.relu = relu;
+    a.BN = plan.BN;
+    a.n_tiles = plan.n_tiles;
+    a.stages = plan.stages;
+    int cols = 32;
+    while (cols < 2 * plan.BN) cols <<= 1;
+    a.tmem_cols = cols;
+    a.vec_out = (g.C_out % 8 == 0 && (reinterpret_cast<uintptr_t>(y) & 15) == 0) ? 1 : 0;
+
+    long long tiles = ((long long)g.M + BM - 1) / BM * plan.n_tiles;
+    int grid = (int)(tiles < num_sms ? tiles : num_sms);
+    if (grid < 1) grid = 1;
+    auto kern = plan.vec ? masked_conv_sm100_kernel<true> : masked_conv_sm100_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, NUM_THREADS, plan.smem_bytes, st>>>(tmap_w, g, a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_repack_w(const void* w, void* wp, int C_out, int K, int Kw, cudaStream_t st)
+{
+    const long long total = (long long)C_out * Kw;
+    int blocks = (int)((total + 255) / 256 < 1024 ? (total + 255) / 256 : 1024);
+    if (blocks < 1) blocks = 1;
+    repack_w_kernel<<<blocks, 256, 0, st>>>(static_cast<const unsigned short*>(w),
+                                            static_cast<unsigned short*>(wp), C_out, K, Kw);
+    return cudaGetLastError();
+}
+
+}  // namespace asx
