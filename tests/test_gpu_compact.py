@@ -1,0 +1,53 @@
+"""S1 on the GPU: the kept-row list must equal the oracle's bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2309_06626_b200 as asx
+
+pytestmark = pytest.mark.gpu
+
+
+def _compact(mask_np, offset=0):
+    buf = torch.zeros(mask_np.size + offset + 16, dtype=torch.uint8, device="cuda")
+    view = buf[offset:offset + mask_np.size]
+    view.copy_(torch.from_numpy(mask_np))
+    kept, count, scratch = asx.compact_mask(view)
+    assert asx.lib().asx_compact_status(scratch.data_ptr(), int(torch.cuda.current_stream().cuda_stream)) == 0
+    c = int(count.item())
+    return kept[:c].cpu().numpy(), c
+
+
+@pytest.mark.parametrize("rows", [0, 1, 15, 16, 17, 4095, 4096, 4097, 12544, 100352, 1638400, 5_000_003])
+@pytest.mark.parametrize("q", [0.0, 0.5, 0.9, 1.0])
+def test_compaction_matches_oracle(rows, q):
+    rng = np.random.default_rng(rows + int(q * 10))
+    mask = (rng.random(rows) < q).astype(np.uint8)
+    kept, c = _compact(mask)
+    ref = oracle.kept_list(mask)
+    assert c == ref.size
+    assert np.array_equal(kept, ref)
+
+
+def test_compaction_unaligned_pointer_and_nonbinary_bytes():
+    rng = np.random.default_rng(3)
+    mask = rng.integers(0, 3, 50001).astype(np.uint8)        # 0, 1 or 2: non-zero keeps
+    for off in (1, 7, 8):
+        kept, c = _compact(mask, offset=off)
+        assert np.array_equal(kept, oracle.kept_list(mask))
+
+
+def test_compaction_repeated_calls_share_scratch():
+    mask = (np.random.default_rng(9).random(300000) < 0.3).astype(np.uint8)
+    md = torch.from_numpy(mask).cuda()
+    kept = torch.empty(mask.size, dtype=torch.int32, device="cuda")
+    count = torch.empty(1, dtype=torch.int32, device="cuda")
+    nbytes = asx.lib().asx_compact_scratch_bytes(mask.size)
+    scratch = torch.full(((nbytes + 7) // 8,), -1, dtype=torch.int64, device="cuda")   # dirty on entry
+    st = int(torch.cuda.current_stream().cuda_stream)
+    for _ in range(3):
+        assert asx.lib().asx_compact(md.data_ptr(), mask.size, kept.data_ptr(), count.data_ptr(),
+                                     scratch.data_ptr(), scratch.numel() * 8, st) == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(kept[:int(count.item())].cpu().numpy(), oracle.kept_list(mask))
