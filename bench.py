@@ -1,0 +1,428 @@
+#!/usr/bin/env python
+"""Benchmark of the masked conv-GEMM path on synthetic layer stacks.
+
+One step = one pass of the whole path (mask compaction, implicit-im2col gather, tensor-core
+GEMM on the kept rows, bias+ReLU scatter epilogue with zero fill) over every layer of the
+workload, through the C-ABI library.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 3] [--impl ours|reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs its own replica of the
+batch (lowered rows are independent: the batch is split across GPUs, there is no collective
+on the data path); the timed region is bracketed by barriers and the maximum over ranks is
+reported.  `--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "masked conv-GEMM actual TFLOP/s"
+L2_BYTES = 126 * 1024 * 1024
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def workload_name(cfg: int) -> str:
+    return {1: "single 3x3 conv 56x56x64->64 bs1, 50% rows dropped, block 1",
+            2: "ResNet-18 conv stack 224x224 bs1, 30% row sparsity, block 1",
+            3: "ResNet-18 conv stack 224x224 bs64, 50% row sparsity, block 4",
+            4: "CSP-Darknet-like conv stack 640x640 bs16, 40% row sparsity, block 2",
+            5: "3x3 conv 28x28x256->256 bs128 sparsity/block sweep"}[cfg]
+
+
+# --------------------------------------------------------------------------------------------
+# clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.thread, self.idx = [], None, None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = [r for r in self.rows if t0 <= r[0] <= t1] or self.rows
+        for _, line in rows:
+            f = [c.strip() for c in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------
+# the CPU oracle leg (cpu_baseline and --impl reference)
+def oracle_problems(cfg: int):
+    probs = []
+    for spec in wl.config(cfg):
+        s1 = wl.with_batch(spec, 1)          # the first image of the batch; same seeds
+        probs.append((s1, wl.make_x(s1), wl.make_w(s1), wl.make_b(s1), wl.make_layer_mask(s1)))
+    return probs
+
+
+def oracle_pass(probs, frac: float):
+    """Runs the oracle on the first ceil(frac*P) output positions of image 0 of every layer.
+    Returns (seconds, kept FLOPs)."""
+    import oracle
+    flops, t0 = 0, time.perf_counter()
+    for s, x, w, b, m in probs:
+        n = max(1, int(np.ceil(frac * s.P)))
+        sel = np.arange(n, dtype=np.int64)
+        oracle.masked_conv_rows(x, w, b, m, s.stride, s.pad, True, sel)
+        flops += 2 * int(m[:n].sum()) * s.K * s.N
+    return time.perf_counter() - t0, flops
+
+
+def cpu_baseline(cfg: int, budget_s: float = 15.0):
+    import oracle
+    oracle.build()
+    probs = oracle_problems(cfg)
+    t_cal, _ = oracle_pass(probs, 1.0)
+    reps = int(max(1, min(64, budget_s / max(t_cal, 1e-3))))
+    t, f = 0.0, 0
+    for _ in range(reps):
+        dt, df = oracle_pass(probs, 1.0)
+        t += dt; f += df
+    return {"value": f / t / 1e12, "unit": "TFLOP/s", "cores": oracle.n_threads(), "kind": "oracle",
+            "sample": f"image 0 of every layer of the workload, all output rows, {reps} passes "
+                      f"({f / 1e9:.1f} GFLOP kept, {t:.1f} s)"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    oracle.build()
+    probs = oracle_problems(args.config)
+    t_cal, _ = oracle_pass(probs, 1.0)
+    target = 120.0 / max(1, args.steps + args.warmup)
+    frac = min(1.0, target / max(t_cal, 1e-3))
+    for _ in range(args.warmup):
+        oracle_pass(probs, frac)
+    t, f = 0.0, 0
+    for _ in range(args.steps):
+        dt, df = oracle_pass(probs, frac)
+        t += dt; f += df
+    val = f / t / 1e12
+    sample = (f"per step: the first {frac * 100:.2f}% of the output rows of image 0 of every layer "
+              f"({f / args.steps / 1e9:.3f} GFLOP kept)")
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": workload_name(args.config)},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.n_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# --------------------------------------------------------------------------------------------
+# the GPU leg
+class DeviceLayer:
+    def __init__(self, spec, torch, asx, dense_twin=True):
+        self.spec = spec
+        x, w, b = wl.make_x(spec), wl.make_w(spec), wl.make_b(spec)
+        self.mask = wl.make_layer_mask(spec)
+        self.x_host = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+        self.x = self.x_host.cuda()
+        self.w = torch.from_numpy(w).to(torch.bfloat16).cuda()
+        self.b = torch.from_numpy(b).cuda()
+        self.y = torch.empty((spec.Nb, spec.Ho, spec.Wo, spec.C_out), dtype=torch.bfloat16, device="cuda")
+        self.y_host = torch.empty(self.y.shape, dtype=torch.bfloat16).pin_memory()
+        self.layer = asx.MaskedConvLayer(spec.C_in, spec.C_out, spec.kh, spec.kw, spec.stride, spec.pad)
+        self.layer.set_mask(self.mask)
+        self.dense = None
+        if dense_twin:
+            self.dense = asx.MaskedConvLayer(spec.C_in, spec.C_out, spec.kh, spec.kw, spec.stride, spec.pad)
+            self.dense.set_mask(np.ones(spec.P, np.uint8))
+        kept_rows = int(self.mask.sum()) * spec.Nb
+        self.kept_rows = kept_rows
+        self.flops = wl.algorithmic_flops(spec, kept_rows)
+        self.flops_dense = wl.algorithmic_flops(spec, spec.M)
+        self.bytes = wl.algorithmic_bytes(spec, self.mask)
+        self.ptrs = (self.x.data_ptr(), spec.Nb, spec.H, spec.W, self.w.data_ptr(), self.b.data_ptr(),
+                     self.y.data_ptr())
+        self.launches = 2 + (1 if spec.C_in % 8 else 0)      # compaction, main kernel, filter repack
+
+    def step(self, st, flags, layer=None):
+        L = layer or self.layer
+        rc = L.recompact_raw(st)
+        rc |= L.run_raw(*self.ptrs, flags, st)
+        if rc:
+            raise RuntimeError(f"asx call failed with status {rc} on {self.spec.name}")
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2309_06626_b200 as asx
+    from paper_2309_06626_b200 import build as asx_build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        asx_build.build()
+    if world > 1:
+        dist.barrier()
+    asx.lib()
+    peaks = load_peaks()
+    st_obj = torch.cuda.current_stream()
+    st = int(st_obj.cuda_stream)
+    RELU = asx.ACT_RELU
+
+    specs = wl.config(args.config)
+    layers = [DeviceLayer(s, torch, asx) for s in specs]
+    torch.cuda.synchronize()
+    footprint = sum(L.x.numel() * 2 + L.y.numel() * 2 + L.w.numel() * 2 for L in layers)
+
+    def one_step(dense=False):
+        for L in layers:
+            L.step(st, RELU, L.dense if dense else None)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    barrier()
+
+    # ---- timed region: K steps, device time by CUDA events on the launching stream
+    K = args.steps
+    n_probe = min(K, 40)                                    # steps that also time each main-kernel launch
+    probe_steps = set(np.linspace(0, K - 1, n_probe).astype(int).tolist())
+    probe_events = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    e0.record(st_obj)
+    for k in range(K):
+        if k in probe_steps:
+            row = []
+            for L in layers:
+                rc = L.layer.recompact_raw(st)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(st_obj)
+                rc |= L.layer.run_raw(*L.ptrs, RELU, st)
+                b.record(st_obj)
+                if rc:
+                    raise RuntimeError(f"asx call failed with status {rc}")
+                row.append((a, b))
+            probe_events.append(row)
+        else:
+            one_step()
+    e1.record(st_obj)
+    barrier()
+    t_wall1 = time.time()
+    ms_total = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / K
+    for L in layers:
+        if L.layer.device_status() != 0:
+            raise RuntimeError("a kernel reported a bounded-wait timeout")
+
+    flops_step = sum(L.flops for L in layers)
+    dense_flops_step = sum(L.flops_dense for L in layers)
+    value = world * flops_step / (ms_step * 1e-3) / 1e12
+
+    # main-kernel durations (dominant kernel), per layer, averaged over the probed steps
+    per_layer_ms = [statistics.mean(row[i][0].elapsed_time(row[i][1]) for row in probe_events)
+                    for i in range(len(layers))]
+    kern_ms = sum(per_layer_ms)
+    achieved = flops_step / (kern_ms * 1e-3) / 1e12
+    peak_tf = peaks["bf16_tflops_sustained"]
+    roof_ms = sum(max(L.flops / (peaks["bf16_tflops"] * 1e12), L.bytes / (peaks["hbm_gbs"] * 1e9)) * 1e3
+                  for L in layers)
+
+    # ---- the same kernels at sparsity 0 (all-ones masks), and cuDNN dense convolution
+    K0 = max(3, min(K, 100))
+    for _ in range(3):
+        one_step(dense=True)
+    torch.cuda.synchronize()
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    d0.record(st_obj)
+    for _ in range(K0):
+        one_step(dense=True)
+    d1.record(st_obj)
+    torch.cuda.synchronize()
+    ms_dense = d0.elapsed_time(d1) / K0
+
+    cudnn_ms = None
+    if rank == 0 and not args.no_cudnn:
+        import torch.nn.functional as F
+        views = [(L.x.permute(0, 3, 1, 2), L.w.permute(0, 3, 1, 2), L.b.to(torch.bfloat16), L.spec) for L in layers]
+
+        def cudnn_step():
+            for xv, wv, bv, s in views:
+                F.conv2d(xv, wv, bv, stride=s.stride, padding=s.pad)
+        for _ in range(3):
+            cudnn_step()
+        torch.cuda.synchronize()
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record(st_obj)
+        for _ in range(K0):
+            cudnn_step()
+        c1.record(st_obj)
+        torch.cuda.synchronize()
+        cudnn_ms = c0.elapsed_time(c1) / K0
+
+    # ---- end to end: host buffers, H2D of every layer's input and D2H of every output inside the timed region
+    Ke = max(3, min(K, 10))
+    h2d = sum(L.x_host.numel() * 2 for L in layers)
+    d2h = sum(L.y_host.numel() * 2 for L in layers)
+
+    def e2e_step():
+        for L in layers:
+            L.x.copy_(L.x_host, non_blocking=True)
+            L.step(st, RELU)
+            L.y_host.copy_(L.y, non_blocking=True)
+    e2e_step()
+    barrier()
+    tw0 = time.perf_counter()
+    for _ in range(Ke):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - tw0) * 1e3 / Ke
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_val = world * flops_step / (e2e_ms * 1e-3) / 1e12
+    t_gpu_end = time.time()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+    sampler.stop()
+    clocks = sampler.summary(t_wall0, t_wall1)
+    clocks_all = sampler.summary(0, t_gpu_end)
+    if clocks["samples"] < 2:
+        clocks = clocks_all
+    cpu = None if args.no_cpu_baseline else cpu_baseline(args.config)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": K,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload_name(args.config), "layers": len(layers),
+                   "l2": f"inputs larger than L2: each step cycles {footprint / 1e6:.0f} MB of distinct "
+                         f"layer buffers (L2 is {L2_BYTES / 1e6:.0f} MB)",
+                   "step": "per layer: mask compaction + fused gather/GEMM/scatter kernel",
+                   "mask": "one mask per layer shared by the batch"},
+        "dense_equivalent_tflops": world * dense_flops_step / (ms_step * 1e-3) / 1e12,
+        "speedup_vs_sparsity0": ms_dense / ms_step,
+        "ms_per_step_sparsity0": ms_dense,
+        "speedup_vs_cudnn_dense": (cudnn_ms / ms_step) if cudnn_ms else None,
+        "cudnn_dense_ms_per_step": cudnn_ms,
+        "clocks": clocks,
+        "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms},
+        "gpu_launches": K * sum(L.launches for L in layers),
+        "roofline": {"bound": "tensor", "kernel": "masked_conv_sm100_kernel", "achieved": achieved,
+                     "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": None,
+                     "peak_source": f"{peaks['source']} (sustained bf16 matmul; burst {peaks['bf16_tflops']})",
+                     "kernel_ms_per_step": kern_ms,
+                     "frac_of_layer_roofs": roof_ms / kern_ms,
+                     "layer_roofs_ms_per_step": roof_ms},
+        "cpu_baseline": cpu,
+        "per_layer": [{"name": L.spec.name, "M": L.spec.M, "K": L.spec.K, "N": L.spec.N, "kept_rows": L.kept_rows,
+                       "ms": per_layer_ms[i], "tflops": L.flops / (per_layer_ms[i] * 1e-3) / 1e12,
+                       "gbs": L.bytes / (per_layer_ms[i] * 1e-3) / 1e9}
+                      for i, L in enumerate(layers)],
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cudnn", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

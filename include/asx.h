@@ -94,6 +94,13 @@ asx_status asx_set_mask_random(asx_layer* layer, int64_t rows, double sparsity, 
                                uint64_t seed, void* cuda_stream);
 
 /*
+ * Rebuild the kept-row list from the stored mask (stage i alone; the same work the
+ * ASX_RECOMPACT flag does inside asx_run).  Asynchronous on `cuda_stream`; allocates nothing.
+ * ASX_ERR_NO_MASK before any asx_set_mask*.
+ */
+asx_status asx_recompact(asx_layer* layer, void* cuda_stream);
+
+/*
  * Run the layer (Section 3.2 stages i-iii fused): gather the kept windows of x, multiply by
  * the filters on the tensor cores, add the bias, apply the activation, write kept rows to
  * their NHWC positions and zeros to the dropped ones.  Every element of y is written once.

@@ -13,7 +13,7 @@ ACT_RELU, RECOMPACT, IMPL_NAIVE = 1, 2, 4
 
 # every symbol include/asx.h declares
 EXPORTS = (
-    "asx_status_string", "asx_create_layer", "asx_set_mask", "asx_set_mask_random", "asx_run",
+    "asx_status_string", "asx_create_layer", "asx_set_mask", "asx_set_mask_random", "asx_recompact", "asx_run",
     "asx_get_kept", "asx_get_kept_host", "asx_get_mask", "asx_last_device_status", "asx_destroy",
     "asx_compact_scratch_bytes", "asx_compact", "asx_compact_status",
 )
@@ -44,6 +44,7 @@ def lib():
         L.asx_create_layer.argtypes = [ci] * 6 + [ctypes.POINTER(vp)]
         L.asx_set_mask.argtypes = [vp, vp, i64, vp]
         L.asx_set_mask_random.argtypes = [vp, i64, ctypes.c_double, ci, ctypes.c_uint64, vp]
+        L.asx_recompact.argtypes = [vp, vp]
         L.asx_run.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, ci, vp]
         L.asx_get_kept.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(vp)]
         L.asx_get_kept_host.argtypes = [vp, vp, i64, ctypes.POINTER(i64)]
@@ -102,6 +103,12 @@ class MaskedConvLayer:
     def set_mask_random(self, rows: int, sparsity: float, block: int, seed: int, stream=None) -> None:
         _check(lib().asx_set_mask_random(self._h, rows, float(sparsity), block, seed, _stream_ptr(stream)),
                "asx_set_mask_random")
+
+    def recompact(self, stream=None) -> None:
+        _check(lib().asx_recompact(self._h, _stream_ptr(stream)), "asx_recompact")
+
+    def recompact_raw(self, stream_ptr: int) -> int:
+        return lib().asx_recompact(self._h, stream_ptr)
 
     def run(self, x, w, bias=None, out=None, flags: int = ACT_RELU, stream=None):
         """x: CUDA bf16 [Nb][H][W][C_in]; w: CUDA bf16 [C_out][kh][kw][C_in]; bias: CUDA fp32 or

@@ -215,6 +215,16 @@ asx_status asx_set_mask_random(asx_layer* L, int64_t rows, double sparsity, int 
     return asx_set_mask(L, mask.data(), rows, cuda_stream);
 }
 
+asx_status asx_recompact(asx_layer* L, void* cuda_stream)
+{
+    if (L == nullptr) return ASX_ERR_INVALID_ARG;
+    if (!L->has_mask) return ASX_ERR_NO_MASK;
+    const asx_status s = bind_device(L);
+    if (s != ASX_OK) return s;
+    L->last_stream = static_cast<cudaStream_t>(cuda_stream);
+    return run_compaction(L, L->last_stream);
+}
+
 asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void* w, const float* bias,
                    void* y, int flags, void* cuda_stream)
 {
