@@ -12,11 +12,10 @@
 //   MMA thread      issues tcgen05.mma (128 x BN x 16, bf16 -> fp32) into one of two
 //                   accumulators in tensor memory, so the epilogue of tile i overlaps the
 //                   main loop of tile i+1.
-//   epilogue warps  first write zeros to the dropped output rows that lie between this
-//                   tile's first kept row and the next tile's first kept row (kept rows are
-//                   ascending, so these intervals partition the output), then read the
-//                   accumulator, add the bias, apply ReLU, round to bf16 and store each kept
-//                   row at its NHWC position.  Every output element is written exactly once.
+//   epilogue warps  read the accumulator, add the bias, apply ReLU, round to bf16 and store
+//                   each kept row at its NHWC position.
+//   zero warps      write zeros to the dropped rows of this block's share of the output,
+//                   straight from the mask.  Every output element is written exactly once.
 //
 // The kept-row count is read from device memory, so the host never has to know it.
 // All waits are bounded: a wait that runs out sets the status word and every role leaves.
@@ -32,10 +31,13 @@ constexpr int BM = 128;                 // kept rows per tile (UMMA M)
 constexpr int BK = 64;                  // K elements per pipeline stage (one 128-byte swizzled row)
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int MAX_STAGES = 8;
-constexpr int LAG = 2;                  // cp.async groups a producer thread keeps in flight
+constexpr int MIN_STAGES = 4;
 constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_EPI0 = 2, WARP_PROD0 = 6;
-constexpr int NUM_PROD_WARPS = 4, NUM_EPI_WARPS = 4;
-constexpr int NUM_THREADS = 32 * (WARP_PROD0 + NUM_PROD_WARPS);
+constexpr int NUM_PROD_WARPS = 8, NUM_EPI_WARPS = 4;
+constexpr int ROWS_PER_PASS = NUM_PROD_WARPS * 4;     // rows one producer instruction covers
+constexpr int PASSES = BM / ROWS_PER_PASS;            // rows per producer thread and stage
+constexpr int WARP_ZERO0 = WARP_PROD0 + NUM_PROD_WARPS, NUM_ZERO_WARPS = 2;
+constexpr int NUM_THREADS = 32 * (WARP_ZERO0 + NUM_ZERO_WARPS);
 constexpr long long WAIT_CYCLE_LIMIT = 4000000000ll;   // about two seconds
 
 struct FastArgs {
@@ -52,6 +54,7 @@ struct FastArgs {
 };
 
 struct Shared {           // lives after the operand stages
+    float bias[2][256];   // bias of the tile's columns, double buffered
     unsigned long long full[MAX_STAGES];
     unsigned long long empty[MAX_STAGES];
     unsigned long long acc_full[2];
@@ -129,7 +132,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1 + NUM_PROD_WARPS);
+            ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1 + NUM_PROD_WARPS * 32);
             ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), 1);
         }
         for (int i = 0; i < 2; ++i) {
@@ -185,6 +188,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
                     const int s = it % S;
                     const uint32_t ph = (uint32_t)(it / S) & 1u;
                     if (!wait_bar(ptx::smem_u32(&sh->full[s]), ph, abort_flag, a.dev_status)) { ok = false; break; }
+                    ptx::fence_proxy_async_smem();      // the gathered rows were written through the generic proxy
                     ptx::tc_fence_after_sync();
                     const uint32_t a_addr = smem_base + s * stage_bytes;
                     const uint64_t adesc = ptx::umma_desc_k_major_sw128(a_addr);
@@ -200,79 +204,67 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
     } else if (warp < WARP_PROD0) {
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3;                       // TMEM lanes 32q .. 32q+31 belong to this warp
-        const int et = (warp - WARP_EPI0) * 32 + lane;
         unsigned short* y2 = reinterpret_cast<unsigned short*>(a.y);
         int ti = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
             const int m_tile = t / a.n_tiles, n_tile = t - m_tile * a.n_tiles;
             const int n0 = n_tile * BN;
-            const int ncols = min(N - n0, BN);
-            // zeros for the dropped rows this tile owns
-            {
-                const int lo = (m_tile == 0) ? 0 : out_row_of(m_tile * BM, cnt, g, a.kept);
-                const int hi = (m_tile == m_tiles - 1) ? g.M : out_row_of((m_tile + 1) * BM, cnt, g, a.kept);
-                if (a.vec_out) {
-                    const int cpr = ncols >> 3;
-                    const long long total = (long long)(hi - lo) * cpr;
-                    for (long long i = et; i < total; i += NUM_EPI_WARPS * 32) {
-                        const int rr = (int)(i / cpr), cc = (int)(i - (long long)rr * cpr);
-                        const int row = lo + rr;
-                        const int p = (g.rows == g.P) ? row % g.P : row;
-                        if (__ldg(a.mask + p) == 0)
-                            *reinterpret_cast<uint4*>(y2 + (long long)row * N + n0 + cc * 8) = make_uint4(0, 0, 0, 0);
-                    }
-                } else {
-                    const long long total = (long long)(hi - lo) * ncols;
-                    for (long long i = et; i < total; i += NUM_EPI_WARPS * 32) {
-                        const int rr = (int)(i / ncols), cc = (int)(i - (long long)rr * ncols);
-                        const int row = lo + rr;
-                        const int p = (g.rows == g.P) ? row % g.P : row;
-                        if (__ldg(a.mask + p) == 0) y2[(long long)row * N + n0 + cc] = 0;
-                    }
-                }
-            }
             // kept rows from the accumulator
             const int buf = ti & 1;
             const uint32_t use = (uint32_t)(ti >> 1) & 1u;
             const int rk = m_tile * BM + q * 32 + lane;
             const bool valid = rk < Mk;
             const long long yoff = valid ? (long long)out_row_of(rk, cnt, g, a.kept) * N : 0;
+            {
+                float* sb = sh->bias[buf];
+                const int et = (warp - WARP_EPI0) * 32 + lane;
+                for (int c1 = et; c1 < BN; c1 += NUM_EPI_WARPS * 32)
+                    sb[c1] = (a.bias != nullptr && n0 + c1 < N) ? __ldg(a.bias + n0 + c1) : 0.f;
+                asm volatile("bar.sync 1, %0;" ::"n"(NUM_EPI_WARPS * 32) : "memory");
+            }
+            const float* sbias = sh->bias[buf];
             if (!wait_bar(ptx::smem_u32(&sh->acc_full[buf]), use, abort_flag, a.dev_status)) { ok = false; break; }
             ptx::tc_fence_after_sync();
             const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
-            for (int c0 = 0; c0 < BN; c0 += 16) {
+            for (int c0 = 0; c0 < BN; c0 += 32) {
                 const int col0 = n0 + c0;
                 if (col0 >= N) break;
-                uint32_t r[16];
-                ptx::tmem_ld_16(tacc + (uint32_t)c0, r);
+                uint32_t r[32];
+                const bool wide = (c0 + 32 <= BN);
+                if (wide) {
+                    ptx::tmem_ld_32(tacc + (uint32_t)c0, r);
+                } else {
+                    uint32_t r16[16];
+                    ptx::tmem_ld_16(tacc + (uint32_t)c0, r16);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) { r[j] = r16[j]; r[16 + j] = 0; }
+                }
                 ptx::tmem_ld_wait();
                 if (valid) {
-                    float v[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int col = col0 + j;
-                        float f = __uint_as_float(r[j]);
-                        if (a.bias != nullptr && col < N) f += __ldg(a.bias + col);
-                        v[j] = a.relu ? fmaxf(f, 0.f) : f;
-                    }
-                    if (a.vec_out) {
+                    for (int h = 0; h < 4; ++h) {
+                        const int colh = col0 + 8 * h;
+                        if (colh >= N) break;
+                        float v[8];
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            if (col0 + 8 * h < N) {
-                                uint4 o;
-                                o.x = pack_bf16(v[8 * h + 0], v[8 * h + 1]);
-                                o.y = pack_bf16(v[8 * h + 2], v[8 * h + 3]);
-                                o.z = pack_bf16(v[8 * h + 4], v[8 * h + 5]);
-                                o.w = pack_bf16(v[8 * h + 6], v[8 * h + 7]);
-                                *reinterpret_cast<uint4*>(y2 + yoff + col0 + 8 * h) = o;
-                            }
+                        for (int j = 0; j < 8; ++j) {
+                            float f = __uint_as_float(r[8 * h + j]);
+                            f += sbias[c0 + 8 * h + j];
+                            v[j] = a.relu ? fmaxf(f, 0.f) : f;
                         }
-                    } else {
+                        if (a.vec_out) {
+                            uint4 o;
+                            o.x = pack_bf16(v[0], v[1]);
+                            o.y = pack_bf16(v[2], v[3]);
+                            o.z = pack_bf16(v[4], v[5]);
+                            o.w = pack_bf16(v[6], v[7]);
+                            *reinterpret_cast<uint4*>(y2 + yoff + colh) = o;
+                        } else {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (col0 + j < N)
-                                y2[yoff + col0 + j] = __bfloat16_as_ushort(__float2bfloat16_rn(v[j]));
+                            for (int j = 0; j < 8; ++j)
+                                if (colh + j < N) y2[yoff + colh + j] = __bfloat16_as_ushort(__float2bfloat16_rn(v[j]));
+                        }
                     }
                 }
             }
@@ -280,25 +272,92 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[buf]));
         }
+    } else if (warp >= WARP_ZERO0) {
+        // ------------------------------------------------------------------ zeros for dropped rows
+        // Algorithm 2's post-processing writes zeros wherever the mask is 0.  These warps stream
+        // over this block's share of the output rows, independent of the tile loop: a warp reads
+        // 32 mask bytes (one per lane), a ballot gives the dropped rows, and the lanes write those
+        // rows together.  Kept rows are written by the epilogue, so each element is written once.
+        unsigned short* y2 = reinterpret_cast<unsigned short*>(a.y);
+        const long long lo = (long long)g.M * blockIdx.x / gridDim.x;
+        const long long hi = (long long)g.M * (blockIdx.x + 1) / gridDim.x;
+        const int zw = warp - WARP_ZERO0;
+        const int cpr = N >> 3;                                   // 16-byte chunks per row (vector path)
+        const int rows_per_pass = (a.vec_out && cpr < 32) ? 32 / cpr : 1;
+        const int sub = (a.vec_out && cpr < 32) ? lane / cpr : 0;
+        const int cc = (a.vec_out && cpr < 32) ? lane - sub * cpr : lane;
+        auto is_dropped = [&](long long row) -> bool {
+            if (row >= hi) return false;
+            const int r = (int)row;
+            return __ldg(a.mask + ((g.rows == g.P) ? r % g.P : r)) == 0;
+        };
+        long long base = lo + zw * 32;
+        bool d0 = is_dropped(base + lane);
+        bool d1 = is_dropped(base + NUM_ZERO_WARPS * 32 + lane);
+        while (base < hi) {
+            const unsigned dm = __ballot_sync(0xffffffffu, d0);
+            const long long cur = base;
+            base += NUM_ZERO_WARPS * 32;
+            d0 = d1;
+            d1 = is_dropped(base + NUM_ZERO_WARPS * 32 + lane);   // two groups ahead
+            unsigned rest = dm;
+            if (a.vec_out && cpr < 32) {
+                while (rest) {
+                    int mine = -1;                                  // the sub-th dropped row of this pass
+                    for (int q2 = 0; q2 < rows_per_pass && rest; ++q2) {
+                        const int bit = __ffs(rest) - 1;
+                        rest &= rest - 1;
+                        if (q2 == sub) mine = bit;
+                    }
+                    if (mine >= 0 && sub < rows_per_pass)
+                        *reinterpret_cast<uint4*>(y2 + (cur + mine) * N + cc * 8) = make_uint4(0, 0, 0, 0);
+                }
+            } else if (a.vec_out) {
+                while (rest) {
+                    const long long row = cur + __ffs(rest) - 1;
+                    rest &= rest - 1;
+                    for (int c1 = lane; c1 < cpr; c1 += 32)
+                        *reinterpret_cast<uint4*>(y2 + row * N + c1 * 8) = make_uint4(0, 0, 0, 0);
+                }
+            } else {
+                while (rest) {
+                    const long long row = cur + __ffs(rest) - 1;
+                    rest &= rest - 1;
+                    for (int c1 = lane; c1 < N; c1 += 32) y2[row * N + c1] = 0;
+                }
+            }
+        }
     } else {
         // ------------------------------------------------------------------ gather producers
         const int pw = warp - WARP_PROD0;
         const int c = lane & 7;                        // 16-byte chunk of the 128-byte row
-        const int rsub = pw * 4 + (lane >> 3);         // row within each group of 16
+        const int rsub = pw * 4 + (lane >> 3);         // row within each group of ROWS_PER_PASS
         const uint32_t sw_off = (uint32_t)(rsub * 128 + ((c ^ (rsub & 7)) << 4));
         const unsigned short* x2 = reinterpret_cast<const unsigned short*>(a.x);
+        // position of this thread's first K element (k = 8c) in the filter window
+        const int tap0 = (c * 8) / g.C_in, ci0 = c * 8 - tap0 * g.C_in;
+        const int ky0 = tap0 / g.kw, kx0 = tap0 - ky0 * g.kw;
         int it = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        // output rows of the first tile; the next tile's are fetched while the current one streams
+        int orow[PASSES];
+        auto fetch_rows = [&](int t) {
             const int m_tile = t / a.n_tiles;
-            int pix[8], iy0[8], ix0[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int rk = m_tile * BM + i * 16 + rsub;
+            for (int i = 0; i < PASSES; ++i) {
+                const int rk = m_tile * BM + i * ROWS_PER_PASS + rsub;
+                orow[i] = (t < total_tiles && rk < Mk) ? out_row_of(rk, cnt, g, a.kept) : -1;
+            }
+        };
+        fetch_rows(blockIdx.x);
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            int pix[PASSES], iy0[PASSES], ix0[PASSES];
+#pragma unroll
+            for (int i = 0; i < PASSES; ++i) {
                 pix[i] = 0; ix0[i] = 0; iy0[i] = -(1 << 24);          // no tap is in bounds
-                if (rk < Mk) {
-                    const int row = out_row_of(rk, cnt, g, a.kept);
-                    if ((unsigned)row < (unsigned)g.M) {
+                const int row = orow[i];
+                if (row >= 0) {
+                    if (row < g.M) {
                         const int n = row / g.P, p = row - n * g.P;
                         const int oy = p / g.Wo, ox = p - oy * g.Wo;
                         iy0[i] = oy * g.stride - g.pad;
@@ -309,44 +368,43 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
                     }
                 }
             }
+            fetch_rows(t + gridDim.x);
+            int ky = ky0, kx = kx0, ci = ci0;          // window position of K element kb*64 + 8c
             for (int kb = 0; kb < KB; ++kb, ++it) {
                 const int s = it % S;
                 const uint32_t ph = (uint32_t)(it / S) & 1u;
                 if (!wait_bar(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
                 const uint32_t dst0 = smem_base + s * stage_bytes + sw_off;
                 if (VEC) {
-                    const int k = kb * BK + c * 8;
-                    const bool kvalid = k < g.K;
-                    const int tap = k / g.C_in, ci = k - tap * g.C_in;
-                    const int ky = tap / g.kw, kx = tap - ky * g.kw;
+                    const bool kvalid = ky < g.kh;     // past K: the window is exhausted
                     const int koff = ky * g.W + kx;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
+                    for (int i = 0; i < PASSES; ++i) {
                         const bool in = kvalid && (unsigned)(iy0[i] + ky) < (unsigned)g.H &&
                                         (unsigned)(ix0[i] + kx) < (unsigned)g.W;
                         const unsigned short* src = in ? x2 + ((long long)(pix[i] + koff) * g.C_in + ci) : x2;
-                        ptx::cp_async_16(dst0 + i * (16 * 128), src, in ? 16u : 0u);
+                        ptx::cp_async_16(dst0 + i * (ROWS_PER_PASS * 128), src, in ? 16u : 0u);
                     }
-                    ptx::cp_async_commit();
-                    if (it >= LAG) {
-                        ptx::cp_async_wait<LAG>();
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->full[(it - LAG) % S]));
+                    ptx::cp_async_mbar_arrive_noinc(ptx::smem_u32(&sh->full[s]));
+                    // advance the window position by 64 K elements
+                    ci += BK;
+                    while (ci >= g.C_in) {
+                        ci -= g.C_in;
+                        if (++kx == g.kw) { kx = 0; ++ky; }
                     }
                 } else {
                     int eoff[8], eky[8], ekx[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         const int k = kb * BK + c * 8 + e;
-                        const int tap = k / g.C_in, ci = k - tap * g.C_in;
-                        const int ky = tap / g.kw;
-                        eky[e] = (k < g.K) ? ky : (1 << 26);                  // past K: never in bounds
-                        ekx[e] = tap - ky * g.kw;
-                        eoff[e] = (ky * g.W + ekx[e]) * g.C_in + ci;
+                        const int tap = k / g.C_in, cie = k - tap * g.C_in;
+                        const int kye = tap / g.kw;
+                        eky[e] = (k < g.K) ? kye : (1 << 26);                 // past K: never in bounds
+                        ekx[e] = tap - kye * g.kw;
+                        eoff[e] = (kye * g.W + ekx[e]) * g.C_in + cie;
                     }
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
+                    for (int i = 0; i < PASSES; ++i) {
                         unsigned short e16[8];
                         const long long base = (long long)pix[i] * g.C_in;
 #pragma unroll
@@ -360,23 +418,14 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
                         v.y = e16[2] | ((uint32_t)e16[3] << 16);
                         v.z = e16[4] | ((uint32_t)e16[5] << 16);
                         v.w = e16[6] | ((uint32_t)e16[7] << 16);
-                        ptx::st_shared_v4(dst0 + i * (16 * 128), v);
+                        ptx::st_shared_v4(dst0 + i * (ROWS_PER_PASS * 128), v);
                     }
                     ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->full[s]));
+                    ptx::mbar_arrive(ptx::smem_u32(&sh->full[s]));
                 }
             }
         }
-        if (VEC) {
-            ptx::cp_async_wait<0>();
-            ptx::fence_proxy_async_smem();
-            __syncwarp();
-            if (ok && lane == 0) {
-                for (int j = (it > LAG ? it - LAG : 0); j < it; ++j)
-                    ptx::mbar_arrive(ptx::smem_u32(&sh->full[j % S]));
-            }
-        }
+        if (VEC) ptx::cp_async_wait<0>();          // nothing of this thread is in flight at exit
     }
 
     ptx::tc_fence_before_sync();
@@ -411,7 +460,7 @@ bool plan_fast(const ConvGeom& g, FastPlan* plan)
     const int budget = 227 * 1024 - 1024 - (int)sizeof(Shared);
     int S = budget / stage_bytes;
     if (S > MAX_STAGES) S = MAX_STAGES;
-    if (S < LAG + 2) return false;
+    if (S < MIN_STAGES) return false;
     plan->BN = BN;
     plan->n_tiles = n_tiles;
     plan->stages = S;
@@ -449,8 +498,12 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     int grid = (int)(tiles < num_sms ? tiles : num_sms);
     if (grid < 1) grid = 1;
     auto kern = plan.vec ? masked_conv_sm100_kernel<true> : masked_conv_sm100_kernel<false>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
-    if (e != cudaSuccess) return e;
+    static int smem_set[2] = {0, 0};            // largest dynamic shared memory size enabled so far
+    if (plan.smem_bytes > smem_set[plan.vec]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
+        if (e != cudaSuccess) return e;
+        smem_set[plan.vec] = plan.smem_bytes;
+    }
     kern<<<grid, NUM_THREADS, plan.smem_bytes, st>>>(tmap_w, g, a);
     return cudaGetLastError();
 }
