@@ -34,10 +34,10 @@ constexpr int MAX_STAGES = 8;
 constexpr int MIN_STAGES = 4;
 constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_EPI0 = 2, WARP_PROD0 = 6;
 constexpr int NUM_PROD_WARPS = 8, NUM_EPI_WARPS = 4;
-constexpr int ROWS_PER_PASS = NUM_PROD_WARPS * 4;     // rows one producer instruction covers
-constexpr int PASSES = BM / ROWS_PER_PASS;            // rows per producer thread and stage
+constexpr int INFO_RING = 8;            // tiles whose row coordinates are kept in shared memory
 constexpr int WARP_ZERO0 = WARP_PROD0 + NUM_PROD_WARPS, NUM_ZERO_WARPS = 2;
-constexpr int NUM_THREADS = 32 * (WARP_ZERO0 + NUM_ZERO_WARPS);
+constexpr int WARP_INFO = WARP_ZERO0 + NUM_ZERO_WARPS;
+constexpr int NUM_THREADS = 32 * (WARP_INFO + 1);
 constexpr long long WAIT_CYCLE_LIMIT = 4000000000ll;   // about two seconds
 
 struct FastArgs {
@@ -54,7 +54,10 @@ struct FastArgs {
 };
 
 struct Shared {           // lives after the operand stages
+    int2 rowinfo[INFO_RING][BM];   // per tile row: first input pixel index, (iy0 << 16) | (ix0 & 0xffff)
     float bias[2][256];   // bias of the tile's columns, double buffered
+    unsigned long long info_full[INFO_RING];
+    unsigned long long info_empty[INFO_RING];
     unsigned long long full[MAX_STAGES];
     unsigned long long empty[MAX_STAGES];
     unsigned long long acc_full[2];
@@ -132,8 +135,12 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1 + NUM_PROD_WARPS * 32);
+            ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1 + 32);        // filter slab + the 32 lanes of one gather warp
             ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), 1);
+        }
+        for (int i = 0; i < INFO_RING; ++i) {
+            ptx::mbar_init(ptx::smem_u32(&sh->info_full[i]), 1);
+            ptx::mbar_init(ptx::smem_u32(&sh->info_empty[i]), (uint32_t)KB);    // one arrival per stage of the tile
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh->acc_full[i]), 1);
@@ -155,28 +162,68 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
     if (warp == WARP_TMA) {
         // ------------------------------------------------------------------ filter slabs by TMA
         if (lane == 0) {
-            int it = 0;
+            int s = 0;
+            uint32_t ph = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 const int n_tile = t % a.n_tiles;
-                for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int s = it % S;
-                    const uint32_t ph = (uint32_t)(it / S) & 1u;
+                for (int kb = 0; kb < KB; ++kb) {
                     if (!wait_bar(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
                     const uint32_t full = ptx::smem_u32(&sh->full[s]);
                     ptx::mbar_arrive_expect_tx(full, (uint32_t)(BN * BK * 2));
                     ptx::tma_load_2d(smem_base + s * stage_bytes + A_STAGE_BYTES, &tmap_w, full, kb * BK, n_tile * BN);
+                    if (++s == S) { s = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {   // let loads already issued land before the block's shared memory goes away
                 for (int i = 0; i < 64; ++i) __nanosleep(1000);
             }
         }
+    } else if (warp == WARP_INFO) {
+        // ------------------------------------------------------------------ row coordinates
+        // Decodes the kept rows of upcoming tiles into the shared-memory ring, four rows per lane,
+        // running ahead of the gather warps by up to INFO_RING tiles.
+        int j = 0;
+        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++j) {
+            const int r = j % INFO_RING;
+            int good = 1;
+            if (lane == 0)
+                good = wait_bar(ptx::smem_u32(&sh->info_empty[r]), ((uint32_t)(j / INFO_RING) & 1u) ^ 1u, abort_flag, a.dev_status) ? 1 : 0;
+            good = __shfl_sync(0xffffffffu, good, 0);
+            if (!good) break;
+            const int m_tile = t / a.n_tiles;
+            int orow[4];
+#pragma unroll
+            for (int q2 = 0; q2 < 4; ++q2) {
+                const int rk = m_tile * BM + lane * 4 + q2;
+                orow[q2] = (rk < Mk) ? out_row_of(rk, cnt, g, a.kept) : -1;
+            }
+#pragma unroll
+            for (int q2 = 0; q2 < 4; ++q2) {
+                int2 info = make_int2(0, (int)0x80000000u);            // iy0 = -32768: no tap is in bounds
+                const int row = orow[q2];
+                if (row >= 0) {
+                    if (row < g.M) {
+                        const int n = row / g.P, p = row - n * g.P;
+                        const int oy = p / g.Wo, ox = p - oy * g.Wo;
+                        const int iy0 = oy * g.stride - g.pad, ix0 = ox * g.stride - g.pad;
+                        info.x = (n * g.H + iy0) * g.W + ix0;
+                        info.y = (iy0 << 16) | (ix0 & 0xffff);
+                    } else {
+                        atomicOr(a.dev_status, DEV_BAD_INDEX);
+                    }
+                }
+                sh->rowinfo[r][lane * 4 + q2] = info;
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_full[r]));
+        }
     } else if (warp == WARP_MMA) {
         // ------------------------------------------------------------------ MMA issue
         if (lane == 0) {
             const uint32_t idesc = ptx::umma_idesc_bf16(BM, BN);
-            int it = 0, ti = 0;
+            int s = 0, ti = 0;
+            uint32_t ph = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
                 const int buf = ti & 1;
@@ -184,9 +231,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
                 if (!wait_bar(ptx::smem_u32(&sh->acc_empty[buf]), use ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
                 const uint32_t d = tmem_base + (uint32_t)(buf * BN);
-                for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int s = it % S;
-                    const uint32_t ph = (uint32_t)(it / S) & 1u;
+                for (int kb = 0; kb < KB; ++kb) {
                     if (!wait_bar(ptx::smem_u32(&sh->full[s]), ph, abort_flag, a.dev_status)) { ok = false; break; }
                     ptx::fence_proxy_async_smem();      // the gathered rows were written through the generic proxy
                     ptx::tc_fence_after_sync();
@@ -197,6 +242,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
                     for (int k = 0; k < BK / 16; ++k)      // 16 K-elements = 32 bytes = 2 descriptor units
                         ptx::umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
                     ptx::umma_commit(ptx::smem_u32(&sh->empty[s]));
+                    if (++s == S) { s = 0; ph ^= 1u; }
                 }
                 if (ok) ptx::umma_commit(ptx::smem_u32(&sh->acc_full[buf]));
             }
@@ -272,7 +318,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[buf]));
         }
-    } else if (warp >= WARP_ZERO0) {
+    } else if (warp >= WARP_ZERO0) {   // (the row-coordinate warp was handled above)
         // ------------------------------------------------------------------ zeros for dropped rows
         // Algorithm 2's post-processing writes zeros wherever the mask is 0.  These warps stream
         // over this block's share of the output rows, independent of the tile loop: a warp reads
@@ -329,101 +375,90 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
         }
     } else {
         // ------------------------------------------------------------------ gather producers
+        // Each warp owns whole pipeline stages (stage it belongs to warp it % NUM_PROD_WARPS), so
+        // the warps work on different stages at the same time.  Within a stage, 8 lanes cover the
+        // 128 bytes of a row and 4 rows are covered per instruction, 32 instructions per stage.
         const int pw = warp - WARP_PROD0;
         const int c = lane & 7;                        // 16-byte chunk of the 128-byte row
-        const int rsub = pw * 4 + (lane >> 3);         // row within each group of ROWS_PER_PASS
-        const uint32_t sw_off = (uint32_t)(rsub * 128 + ((c ^ (rsub & 7)) << 4));
+        const int rq = lane >> 3;                      // row within each group of 4
+        const uint32_t off_even = (uint32_t)(rq * 128 + ((c ^ rq) << 4));               // rows 8m + rq
+        const uint32_t off_odd = (uint32_t)((4 + rq) * 128 + ((c ^ (4 + rq)) << 4));    // rows 8m + 4 + rq
         const unsigned short* x2 = reinterpret_cast<const unsigned short*>(a.x);
-        // position of this thread's first K element (k = 8c) in the filter window
-        const int tap0 = (c * 8) / g.C_in, ci0 = c * 8 - tap0 * g.C_in;
-        const int ky0 = tap0 / g.kw, kx0 = tap0 - ky0 * g.kw;
-        int it = 0;
-        bool ok = true;
-        // output rows of the first tile; the next tile's are fetched while the current one streams
-        int orow[PASSES];
-        auto fetch_rows = [&](int t) {
-            const int m_tile = t / a.n_tiles;
-#pragma unroll
-            for (int i = 0; i < PASSES; ++i) {
-                const int rk = m_tile * BM + i * ROWS_PER_PASS + rsub;
-                orow[i] = (t < total_tiles && rk < Mk) ? out_row_of(rk, cnt, g, a.kept) : -1;
+        int my_tiles = 0;
+        if ((int)blockIdx.x < total_tiles) my_tiles = (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
+        const int total_its = my_tiles * KB;
+        // A parity wait tells phases one apart, not two: a warp must meet every phase of the stage
+        // slots it uses, so no more warps take part than there are stages (it advances by <= S).
+        const int active = S < NUM_PROD_WARPS ? S : NUM_PROD_WARPS;
+        int cur_j = -1;
+        for (int it = pw; it < total_its && pw < active; it += active) {
+            const int j = it / KB, kb = it - j * KB;
+            const int r = j % INFO_RING;
+            const int s = it % S;
+            const uint32_t ph = (uint32_t)(it / S) & 1u;
+            if (j != cur_j) {
+                if (!wait_bar(ptx::smem_u32(&sh->info_full[r]), (uint32_t)(j / INFO_RING) & 1u, abort_flag, a.dev_status)) break;
+                cur_j = j;
             }
-        };
-        fetch_rows(blockIdx.x);
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            int pix[PASSES], iy0[PASSES], ix0[PASSES];
+            if (!wait_bar(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) break;
+            const uint32_t dst_even = smem_base + s * stage_bytes + off_even;
+            const uint32_t dst_odd = smem_base + s * stage_bytes + off_odd;
+            const int2* info = sh->rowinfo[r];
+            if (VEC) {
+                const int k = kb * BK + c * 8;
+                const int tap = k / g.C_in, ci = k - tap * g.C_in;
+                const int ky = tap / g.kw, kx = tap - ky * g.kw;
+                const bool kvalid = k < g.K;
+                const int koff = ky * g.W + kx;
+#pragma unroll 1
+                for (int b = 0; b < BM / 32; ++b) {
+                    int2 ri[8];                         // row coordinates first, then eight copies back to back
 #pragma unroll
-            for (int i = 0; i < PASSES; ++i) {
-                pix[i] = 0; ix0[i] = 0; iy0[i] = -(1 << 24);          // no tap is in bounds
-                const int row = orow[i];
-                if (row >= 0) {
-                    if (row < g.M) {
-                        const int n = row / g.P, p = row - n * g.P;
-                        const int oy = p / g.Wo, ox = p - oy * g.Wo;
-                        iy0[i] = oy * g.stride - g.pad;
-                        ix0[i] = ox * g.stride - g.pad;
-                        pix[i] = (n * g.H + iy0[i]) * g.W + ix0[i];
-                    } else {
-                        atomicOr(a.dev_status, DEV_BAD_INDEX);
+                    for (int u = 0; u < 8; ++u) ri[u] = info[(b * 8 + u) * 4 + rq];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int iy = (ri[u].y >> 16) + ky, ix = (int)(short)(ri[u].y & 0xffff) + kx;
+                        const bool in = kvalid && (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
+                        const unsigned short* src = in ? x2 + ((long long)(ri[u].x + koff) * g.C_in + ci) : x2;
+                        ptx::cp_async_16(((u & 1) ? dst_odd : dst_even) + (uint32_t)(b * 4 + (u >> 1)) * 1024u, src, in ? 16u : 0u);
                     }
                 }
-            }
-            fetch_rows(t + gridDim.x);
-            int ky = ky0, kx = kx0, ci = ci0;          // window position of K element kb*64 + 8c
-            for (int kb = 0; kb < KB; ++kb, ++it) {
-                const int s = it % S;
-                const uint32_t ph = (uint32_t)(it / S) & 1u;
-                if (!wait_bar(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
-                const uint32_t dst0 = smem_base + s * stage_bytes + sw_off;
-                if (VEC) {
-                    const bool kvalid = ky < g.kh;     // past K: the window is exhausted
-                    const int koff = ky * g.W + kx;
+                ptx::cp_async_mbar_arrive_noinc(ptx::smem_u32(&sh->full[s]));
+            } else {
+                int eoff[8], eky[8], ekx[8];
 #pragma unroll
-                    for (int i = 0; i < PASSES; ++i) {
-                        const bool in = kvalid && (unsigned)(iy0[i] + ky) < (unsigned)g.H &&
-                                        (unsigned)(ix0[i] + kx) < (unsigned)g.W;
-                        const unsigned short* src = in ? x2 + ((long long)(pix[i] + koff) * g.C_in + ci) : x2;
-                        ptx::cp_async_16(dst0 + i * (ROWS_PER_PASS * 128), src, in ? 16u : 0u);
-                    }
-                    ptx::cp_async_mbar_arrive_noinc(ptx::smem_u32(&sh->full[s]));
-                    // advance the window position by 64 K elements
-                    ci += BK;
-                    while (ci >= g.C_in) {
-                        ci -= g.C_in;
-                        if (++kx == g.kw) { kx = 0; ++ky; }
-                    }
-                } else {
-                    int eoff[8], eky[8], ekx[8];
+                for (int e = 0; e < 8; ++e) {
+                    const int k = kb * BK + c * 8 + e;
+                    const int tap = k / g.C_in, cie = k - tap * g.C_in;
+                    const int kye = tap / g.kw;
+                    eky[e] = (k < g.K) ? kye : (1 << 26);                 // past K: never in bounds
+                    ekx[e] = tap - kye * g.kw;
+                    eoff[e] = (kye * g.W + ekx[e]) * g.C_in + cie;
+                }
+#pragma unroll 2
+                for (int i = 0; i < BM / 4; ++i) {
+                    const int2 ri = info[i * 4 + rq];
+                    const int iy0 = ri.y >> 16, ix0 = (int)(short)(ri.y & 0xffff);
+                    unsigned short e16[8];
+                    const long long base = (long long)ri.x * g.C_in;
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
-                        const int k = kb * BK + c * 8 + e;
-                        const int tap = k / g.C_in, cie = k - tap * g.C_in;
-                        const int kye = tap / g.kw;
-                        eky[e] = (k < g.K) ? kye : (1 << 26);                 // past K: never in bounds
-                        ekx[e] = tap - kye * g.kw;
-                        eoff[e] = (kye * g.W + ekx[e]) * g.C_in + cie;
+                        const bool in = (unsigned)(iy0 + eky[e]) < (unsigned)g.H &&
+                                        (unsigned)(ix0 + ekx[e]) < (unsigned)g.W;
+                        e16[e] = in ? __ldg(x2 + base + eoff[e]) : (unsigned short)0;
                     }
-#pragma unroll
-                    for (int i = 0; i < PASSES; ++i) {
-                        unsigned short e16[8];
-                        const long long base = (long long)pix[i] * g.C_in;
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            const bool in = (unsigned)(iy0[i] + eky[e]) < (unsigned)g.H &&
-                                            (unsigned)(ix0[i] + ekx[e]) < (unsigned)g.W;
-                            e16[e] = in ? __ldg(x2 + base + eoff[e]) : (unsigned short)0;
-                        }
-                        uint4 v;
-                        v.x = e16[0] | ((uint32_t)e16[1] << 16);
-                        v.y = e16[2] | ((uint32_t)e16[3] << 16);
-                        v.z = e16[4] | ((uint32_t)e16[5] << 16);
-                        v.w = e16[6] | ((uint32_t)e16[7] << 16);
-                        ptx::st_shared_v4(dst0 + i * (ROWS_PER_PASS * 128), v);
-                    }
-                    ptx::fence_proxy_async_smem();
-                    ptx::mbar_arrive(ptx::smem_u32(&sh->full[s]));
+                    uint4 v;
+                    v.x = e16[0] | ((uint32_t)e16[1] << 16);
+                    v.y = e16[2] | ((uint32_t)e16[3] << 16);
+                    v.z = e16[4] | ((uint32_t)e16[5] << 16);
+                    v.w = e16[6] | ((uint32_t)e16[7] << 16);
+                    ptx::st_shared_v4(((i & 1) ? dst_odd : dst_even) + (uint32_t)(i >> 1) * 1024u, v);
                 }
+                ptx::fence_proxy_async_smem();
+                ptx::mbar_arrive(ptx::smem_u32(&sh->full[s]));
             }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));    // this stage no longer reads the row ring
         }
         if (VEC) ptx::cp_async_wait<0>();          // nothing of this thread is in flight at exit
     }

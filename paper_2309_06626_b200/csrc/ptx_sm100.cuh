@@ -52,8 +52,9 @@ __device__ __forceinline__ void fence_proxy_async_smem()
 // 16-byte global -> shared copy; src_bytes == 0 writes 16 zero bytes and reads nothing.
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes)
-                 : "memory");
+    // no "memory" clobber: ordering against the barrier instructions comes from all of them
+    // being volatile asm; ordinary loads may be scheduled across the copy
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes));
 }
 // Arrive on an mbarrier once all cp.async copies this thread has issued so far have landed;
 // the arrival is counted in the barrier's expected count (noinc).
