@@ -22,6 +22,7 @@ struct asx_layer {
     void* d_scratch = nullptr;
     int32_t* d_small = nullptr;        // [0] kept count, [1] status word
     bool has_mask = false;
+    int64_t host_kept = -1;            // kept entries of the mask when it came from the host, else -1
     // staging for filters whose K is not a multiple of 8
     void* d_wpack = nullptr;
     size_t wpack_bytes = 0;
@@ -29,6 +30,9 @@ struct asx_layer {
     CUtensorMap tmap;
     const void* tmap_ptr = nullptr;
     int tmap_BN = 0, tmap_Kw = 0;
+    CUtensorMap tmap_x;                // x as a [pixels][C_in] matrix, for the TMA row gather
+    const void* tmapx_ptr = nullptr;
+    int64_t tmapx_pixels = 0;
     cudaStream_t last_stream = nullptr;
 };
 
@@ -169,7 +173,11 @@ asx_status asx_set_mask(asx_layer* L, const uint8_t* mask, int64_t rows, void* c
     cudaError_t e;
     if (on_device) {
         e = cudaMemcpyAsync(L->d_mask, mask, (size_t)rows, cudaMemcpyDeviceToDevice, st);
+        L->host_kept = -1;
     } else {
+        int64_t kept = 0;                                         // only sizes the tiles (a launch heuristic)
+        for (int64_t i = 0; i < rows; ++i) kept += mask[i] != 0;
+        L->host_kept = kept;
         e = cudaMemcpyAsync(L->d_mask, mask, (size_t)rows, cudaMemcpyHostToDevice, st);
         if (e == cudaSuccess) e = cudaStreamSynchronize(st);      // the caller may free a host mask on return
     }
@@ -275,7 +283,9 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         return from_cuda(launch_naive(g, x, w, bias, y, L->d_mask, L->d_kept, d_count, relu, st));
 
     FastPlan plan;
-    if (!plan_fast(g, &plan)) return ASX_ERR_UNSUPPORTED;
+    long long est_rows = M;                                       // unknown on the host: assume every row kept
+    if (L->host_kept >= 0) est_rows = (L->rows == P) ? L->host_kept * Nb : L->host_kept;
+    if (!plan_fast(g, L->num_sms, est_rows, &plan)) return ASX_ERR_UNSUPPORTED;
     const void* wsrc = w;
     int Kw = g.K;
     if (!plan.vec) {
@@ -307,7 +317,23 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         if (r != CUDA_SUCCESS) return ASX_ERR_CUDA;
         L->tmap_ptr = wsrc; L->tmap_BN = plan.BN; L->tmap_Kw = Kw;
     }
-    return from_cuda(launch_fast(g, plan, L->tmap, x, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
+    if (plan.vec == 2) {
+        const int64_t pixels = (int64_t)Nb * H * W;
+        if (L->tmapx_ptr != x || L->tmapx_pixels != pixels) {
+            EncodeTiledFn enc = encode_tiled_fn();
+            if (enc == nullptr) return ASX_ERR_CUDA;
+            const cuuint64_t dims[2] = {(cuuint64_t)L->C_in, (cuuint64_t)pixels};
+            const cuuint64_t strides[1] = {(cuuint64_t)L->C_in * 2};
+            const cuuint32_t box[2] = {64u, 1u};
+            const cuuint32_t estr[2] = {1u, 1u};
+            const CUresult r = enc(&L->tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims,
+                                   strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return ASX_ERR_CUDA;
+            L->tmapx_ptr = x; L->tmapx_pixels = pixels;
+        }
+    }
+    return from_cuda(launch_fast(g, plan, L->tmap, plan.vec == 2 ? L->tmap_x : L->tmap, x, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
                                  L->num_sms, st));
 }
 

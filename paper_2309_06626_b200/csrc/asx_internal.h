@@ -38,12 +38,13 @@ struct FastPlan {
     int n_tiles;      // ceil(C_out / BN)
     int stages;
     int smem_bytes;
-    int vec;          // 1: C_in % 8 == 0 (16-byte gathers straight from x); 0: element gather
+    int vec;          // gather mode: 0 element loads (any C_in), 1 cp.async 16 B (C_in % 8 == 0),
+                      // 2 TMA row gather (C_in % 64 == 0)
     int Kpad;         // K rounded up to 64
 };
-bool plan_fast(const ConvGeom& g, FastPlan* plan);
+bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, FastPlan* plan);
 cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorMap& tmap_w,
-                        const void* x, const float* bias, void* y, const uint8_t* mask,
+                        const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
                         int num_sms, cudaStream_t st);
 // repack w[C_out][K] into wp[C_out][Kw] (zero padded), for K not a multiple of 8

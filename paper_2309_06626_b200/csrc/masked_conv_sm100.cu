@@ -30,11 +30,12 @@ namespace {
 constexpr int BM = 128;                 // kept rows per tile (UMMA M)
 constexpr int BK = 64;                  // K elements per pipeline stage (one 128-byte swizzled row)
 constexpr int A_STAGE_BYTES = BM * BK * 2;
+static_assert(BK == 64, "the MMA loop issues four K=16 instructions per stage");
 constexpr int MAX_STAGES = 8;
 constexpr int MIN_STAGES = 4;
 constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_EPI0 = 2, WARP_PROD0 = 6;
 constexpr int NUM_PROD_WARPS = 8, NUM_EPI_WARPS = 4;
-constexpr int INFO_RING = 8;            // tiles whose row coordinates are kept in shared memory
+constexpr int INFO_RING = 8;            // tiles whose row coordinates are kept in shared memory (power of two)
 constexpr int WARP_ZERO0 = WARP_PROD0 + NUM_PROD_WARPS, NUM_ZERO_WARPS = 2;
 constexpr int WARP_INFO = WARP_ZERO0 + NUM_ZERO_WARPS;
 constexpr int NUM_THREADS = 32 * (WARP_INFO + 1);
@@ -53,7 +54,7 @@ struct FastArgs {
     int vec_out;        // C_out % 8 == 0 and y 16-byte aligned: 16-byte stores
 };
 
-struct Shared {           // lives after the operand stages
+struct alignas(16) Shared {           // lives after the operand stages
     int2 rowinfo[INFO_RING][BM];   // per tile row: first input pixel index, (iy0 << 16) | (ix0 & 0xffff)
     float bias[2][256];   // bias of the tile's columns, double buffered
     unsigned long long info_full[INFO_RING];
@@ -66,12 +67,17 @@ struct Shared {           // lives after the operand stages
     int abort;
 };
 
+// Bounded wait on an mbarrier phase.  The waiter is suspended by the hardware between polls
+// (and woken when the phase completes), so waiting warps do not take issue slots from the warps
+// that share their scheduler.  SLEEP_NS is kept as a per-call-site label of how relaxed the
+// waiter may be; it scales the suspend-time hint.
+template <int SLEEP_NS>
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                          int* dev_status)
 {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    while (!ptx::mbar_try_wait(bar, parity)) {
+    while (!ptx::mbar_try_wait_suspend(bar, parity, 2000u + 10u * SLEEP_NS)) {
         if (*abort_flag) return false;
         if (clock64() - t0 > WAIT_CYCLE_LIMIT) {
             *abort_flag = 1;
@@ -80,6 +86,17 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
         }
     }
     return true;
+}
+
+// The same wait for a whole converged warp: lane 0 polls, the result is broadcast.  Polling from
+// every lane multiplies the barrier traffic in shared memory by 32 and slows every waiter down.
+template <int SLEEP_NS>
+__device__ __forceinline__ bool warp_wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                              int* dev_status)
+{
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = wait_bar<SLEEP_NS>(bar, parity, abort_flag, dev_status) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
 // Output row (n*P + p) of the rk-th kept lowered row.
@@ -98,9 +115,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-template <bool VEC>
+enum : int { GATHER_ELEM = 0, GATHER_CPASYNC = 1, GATHER_TMA = 2 };
+
+template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvGeom g, const FastArgs a)
+masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
+                         const ConvGeom g, const FastArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -135,12 +155,14 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
-            ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1 + 32);        // filter slab + the 32 lanes of one gather warp
+            // the filter thread's expect_tx arrival (which in TMA mode also announces the gathered
+            // bytes) + in the copy modes every gather lane's arrival
+            ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1 + (MODE == GATHER_TMA ? 0 : NUM_PROD_WARPS * 32));
             ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), 1);
         }
         for (int i = 0; i < INFO_RING; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh->info_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh->info_empty[i]), (uint32_t)KB);    // one arrival per stage of the tile
+            ptx::mbar_init(ptx::smem_u32(&sh->info_empty[i]), NUM_PROD_WARPS);  // one arrival per gather warp
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(ptx::smem_u32(&sh->acc_full[i]), 1);
@@ -153,7 +175,10 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
         ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), (uint32_t)a.tmem_cols);
         ptx::tmem_relinquish();
     }
-    if (warp == WARP_TMA && lane == 0) ptx::prefetch_tensormap(&tmap_w);
+    if (warp == WARP_TMA && lane == 0) {
+        ptx::prefetch_tensormap(&tmap_w);
+        if (MODE == GATHER_TMA) ptx::prefetch_tensormap(&tmap_x);
+    }
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
@@ -168,9 +193,9 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 const int n_tile = t % a.n_tiles;
                 for (int kb = 0; kb < KB; ++kb) {
-                    if (!wait_bar(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
+                    if (!wait_bar<40>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
                     const uint32_t full = ptx::smem_u32(&sh->full[s]);
-                    ptx::mbar_arrive_expect_tx(full, (uint32_t)(BN * BK * 2));
+                    ptx::mbar_arrive_expect_tx(full, (uint32_t)(BN * BK * 2 + (MODE == GATHER_TMA ? A_STAGE_BYTES : 0)));
                     ptx::tma_load_2d(smem_base + s * stage_bytes + A_STAGE_BYTES, &tmap_w, full, kb * BK, n_tile * BN);
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
@@ -188,7 +213,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
             const int r = j % INFO_RING;
             int good = 1;
             if (lane == 0)
-                good = wait_bar(ptx::smem_u32(&sh->info_empty[r]), ((uint32_t)(j / INFO_RING) & 1u) ^ 1u, abort_flag, a.dev_status) ? 1 : 0;
+                good = wait_bar<200>(ptx::smem_u32(&sh->info_empty[r]), ((uint32_t)(j / INFO_RING) & 1u) ^ 1u, abort_flag, a.dev_status) ? 1 : 0;
             good = __shfl_sync(0xffffffffu, good, 0);
             if (!good) break;
             const int m_tile = t / a.n_tiles;
@@ -220,32 +245,43 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
         }
     } else if (warp == WARP_MMA) {
         // ------------------------------------------------------------------ MMA issue
-        if (lane == 0) {
-            const uint32_t idesc = ptx::umma_idesc_bf16(BM, BN);
-            int s = 0, ti = 0;
-            uint32_t ph = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
-                const int buf = ti & 1;
-                const uint32_t use = (uint32_t)(ti >> 1) & 1u;
-                if (!wait_bar(ptx::smem_u32(&sh->acc_empty[buf]), use ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
+        // The whole warp runs the loop so that descriptors and counters stay in uniform registers;
+        // one elected lane issues the tcgen05 instructions (issuing from inside a divergent
+        // single-lane branch costs about 100 cycles per instruction).
+        const uint32_t idesc = ptx::umma_idesc_bf16(BM, BN);
+        const uint64_t adesc0 = ptx::umma_desc_k_major_sw128(smem_base);
+        int s = 0, ti = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
+            const int buf = ti & 1;
+            const uint32_t use = (uint32_t)(ti >> 1) & 1u;
+            ok = warp_wait_bar<0>(ptx::smem_u32(&sh->acc_empty[buf]), use ^ 1u, abort_flag, a.dev_status);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            const uint32_t d = tmem_base + (uint32_t)(buf * BN);
+            for (int kb = 0; kb < KB; ++kb) {
+                ok = warp_wait_bar<0>(ptx::smem_u32(&sh->full[s]), ph, abort_flag, a.dev_status);
+                if (!ok) break;
+                // Only the cp.async gather writes the stage through the generic proxy without a fence
+                // of its own (TMA writes through the async proxy, the element gather fences after
+                // its stores).
+                if (MODE == GATHER_CPASYNC) ptx::fence_proxy_async_smem();
                 ptx::tc_fence_after_sync();
-                const uint32_t d = tmem_base + (uint32_t)(buf * BN);
-                for (int kb = 0; kb < KB; ++kb) {
-                    if (!wait_bar(ptx::smem_u32(&sh->full[s]), ph, abort_flag, a.dev_status)) { ok = false; break; }
-                    ptx::fence_proxy_async_smem();      // the gathered rows were written through the generic proxy
-                    ptx::tc_fence_after_sync();
-                    const uint32_t a_addr = smem_base + s * stage_bytes;
-                    const uint64_t adesc = ptx::umma_desc_k_major_sw128(a_addr);
-                    const uint64_t bdesc = ptx::umma_desc_k_major_sw128(a_addr + A_STAGE_BYTES);
-#pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)      // 16 K-elements = 32 bytes = 2 descriptor units
-                        ptx::umma_bf16(d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                const uint64_t adesc = adesc0 + (uint64_t)(s * (stage_bytes >> 4));   // start-address field
+                const uint64_t bdesc = adesc + (A_STAGE_BYTES >> 4);
+                if (ptx::elect_one()) {
+                    ptx::umma_bf16(d, adesc, bdesc, idesc, kb != 0 ? 1u : 0u);       // 16 K-elements = 32 bytes
+                    ptx::umma_bf16(d, adesc + 2, bdesc + 2, idesc, 1u);             //   = 2 descriptor units
+                    ptx::umma_bf16(d, adesc + 4, bdesc + 4, idesc, 1u);
+                    ptx::umma_bf16(d, adesc + 6, bdesc + 6, idesc, 1u);
                     ptx::umma_commit(ptx::smem_u32(&sh->empty[s]));
-                    if (++s == S) { s = 0; ph ^= 1u; }
                 }
-                if (ok) ptx::umma_commit(ptx::smem_u32(&sh->acc_full[buf]));
+                __syncwarp();
+                if (++s == S) { s = 0; ph ^= 1u; }
             }
+            if (ok && ptx::elect_one()) ptx::umma_commit(ptx::smem_u32(&sh->acc_full[buf]));
+            __syncwarp();
         }
     } else if (warp < WARP_PROD0) {
         // ------------------------------------------------------------------ epilogue
@@ -270,7 +306,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
                 asm volatile("bar.sync 1, %0;" ::"n"(NUM_EPI_WARPS * 32) : "memory");
             }
             const float* sbias = sh->bias[buf];
-            if (!wait_bar(ptx::smem_u32(&sh->acc_full[buf]), use, abort_flag, a.dev_status)) { ok = false; break; }
+            if (!warp_wait_bar<100>(ptx::smem_u32(&sh->acc_full[buf]), use, abort_flag, a.dev_status)) { ok = false; break; }
             ptx::tc_fence_after_sync();
             const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
             for (int c0 = 0; c0 < BN; c0 += 32) {
@@ -375,92 +411,146 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const ConvG
         }
     } else {
         // ------------------------------------------------------------------ gather producers
-        // Each warp owns whole pipeline stages (stage it belongs to warp it % NUM_PROD_WARPS), so
-        // the warps work on different stages at the same time.  Within a stage, 8 lanes cover the
-        // 128 bytes of a row and 4 rows are covered per instruction, 32 instructions per stage.
+        // Every warp takes part in every stage and owns 16 of the tile's 128 rows.  The rows'
+        // coordinates are read from the shared-memory ring once per tile; the k loop then only
+        // forms addresses and issues copies, whose completion is reported to the stage's mbarrier
+        // asynchronously, so the warps run ahead of the tensor core by up to S stages.
         const int pw = warp - WARP_PROD0;
-        const int c = lane & 7;                        // 16-byte chunk of the 128-byte row
-        const int rq = lane >> 3;                      // row within each group of 4
-        const uint32_t off_even = (uint32_t)(rq * 128 + ((c ^ rq) << 4));               // rows 8m + rq
-        const uint32_t off_odd = (uint32_t)((4 + rq) * 128 + ((c ^ (4 + rq)) << 4));    // rows 8m + 4 + rq
         const unsigned short* x2 = reinterpret_cast<const unsigned short*>(a.x);
-        int my_tiles = 0;
-        if ((int)blockIdx.x < total_tiles) my_tiles = (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1;
-        const int total_its = my_tiles * KB;
-        // A parity wait tells phases one apart, not two: a warp must meet every phase of the stage
-        // slots it uses, so no more warps take part than there are stages (it advances by <= S).
-        const int active = S < NUM_PROD_WARPS ? S : NUM_PROD_WARPS;
-        int cur_j = -1;
-        for (int it = pw; it < total_its && pw < active; it += active) {
-            const int j = it / KB, kb = it - j * KB;
-            const int r = j % INFO_RING;
-            const int s = it % S;
-            const uint32_t ph = (uint32_t)(it / S) & 1u;
-            if (j != cur_j) {
-                if (!wait_bar(ptx::smem_u32(&sh->info_full[r]), (uint32_t)(j / INFO_RING) & 1u, abort_flag, a.dev_status)) break;
-                cur_j = j;
-            }
-            if (!wait_bar(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) break;
-            const uint32_t dst_even = smem_base + s * stage_bytes + off_even;
-            const uint32_t dst_odd = smem_base + s * stage_bytes + off_odd;
-            const int2* info = sh->rowinfo[r];
-            if (VEC) {
-                const int k = kb * BK + c * 8;
-                const int tap = k / g.C_in, ci = k - tap * g.C_in;
-                const int ky = tap / g.kw, kx = tap - ky * g.kw;
-                const bool kvalid = k < g.K;
-                const int koff = ky * g.W + kx;
-#pragma unroll 1
-                for (int b = 0; b < BM / 32; ++b) {
-                    int2 ri[8];                         // row coordinates first, then eight copies back to back
+        const int c = lane & 7;                        // 16-byte chunk of the 128-byte row (copy modes)
+        const int rq = lane >> 3;                      // copy modes: rows 16pw + rq + {0,4,8,12}
+        const int oob = g.Nb * g.H * g.W;              // TMA mode: a row index past the tensor reads zeros
+        if (MODE == GATHER_TMA) {
+            // Lanes 0..3 of each warp run the whole loop on their own: each fetches four rows per
+            // stage with one TMA row gather (one 64-channel slice of one filter tap per stage;
+            // padding taps point past the end of the tensor and read zeros).  The bytes are
+            // announced to the stage's barrier by the filter thread, so nothing here needs the
+            // other lanes, and the next stage's row indices are formed before waiting for its slot.
+            if (lane < 4) {
+                int s = 0, j = 0;
+                uint32_t ph = 0;
+                bool ok = true;
+                for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++j) {
+                    const int r = j & (INFO_RING - 1);
+                    if (!wait_bar<100>(ptx::smem_u32(&sh->info_full[r]), (uint32_t)(j / INFO_RING) & 1u, abort_flag, a.dev_status)) break;
+                    const int2* info = sh->rowinfo[r] + 16 * pw + 4 * lane;
+                    const int4 ra = *reinterpret_cast<const int4*>(info);
+                    const int4 rb = *reinterpret_cast<const int4*>(info + 2);
+                    const int pix[4] = {ra.x, ra.z, rb.x, rb.z}, yx[4] = {ra.y, ra.w, rb.y, rb.w};
+                    __syncwarp(0xfu);
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));    // the ring slot is in registers now
+                    int ky = 0, kx = 0, ci = 0;
+                    auto indices = [&](int (&idx)[4]) {
+                        const int koff = ky * g.W + kx;
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) ri[u] = info[(b * 8 + u) * 4 + rq];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int iy = (ri[u].y >> 16) + ky, ix = (int)(short)(ri[u].y & 0xffff) + kx;
-                        const bool in = kvalid && (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
-                        const unsigned short* src = in ? x2 + ((long long)(ri[u].x + koff) * g.C_in + ci) : x2;
-                        ptx::cp_async_16(((u & 1) ? dst_odd : dst_even) + (uint32_t)(b * 4 + (u >> 1)) * 1024u, src, in ? 16u : 0u);
+                        for (int i = 0; i < 4; ++i) {
+                            const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
+                            idx[i] = ((unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W) ? pix[i] + koff : oob;
+                        }
+                    };
+                    int idx[4];
+                    indices(idx);
+                    for (int kb = 0; kb < KB; ++kb) {
+                        if (!wait_bar<20>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
+                        ptx::tma_gather4_2d(smem_base + s * stage_bytes + (uint32_t)(16 * pw + 4 * lane) * 128u, &tmap_x,
+                                            ptx::smem_u32(&sh->full[s]), ci, idx[0], idx[1], idx[2], idx[3]);
+                        ci += BK;                          // next 64 channels, or the next tap
+                        if (ci >= g.C_in) {
+                            ci = 0;
+                            if (++kx == g.kw) { kx = 0; ++ky; }
+                            indices(idx);
+                        }
+                        if (++s == S) { s = 0; ph ^= 1u; }
                     }
                 }
-                ptx::cp_async_mbar_arrive_noinc(ptx::smem_u32(&sh->full[s]));
-            } else {
-                int eoff[8], eky[8], ekx[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int k = kb * BK + c * 8 + e;
-                    const int tap = k / g.C_in, cie = k - tap * g.C_in;
-                    const int kye = tap / g.kw;
-                    eky[e] = (k < g.K) ? kye : (1 << 26);                 // past K: never in bounds
-                    ekx[e] = tap - kye * g.kw;
-                    eoff[e] = (kye * g.W + ekx[e]) * g.C_in + cie;
-                }
-#pragma unroll 2
-                for (int i = 0; i < BM / 4; ++i) {
-                    const int2 ri = info[i * 4 + rq];
-                    const int iy0 = ri.y >> 16, ix0 = (int)(short)(ri.y & 0xffff);
-                    unsigned short e16[8];
-                    const long long base = (long long)ri.x * g.C_in;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const bool in = (unsigned)(iy0 + eky[e]) < (unsigned)g.H &&
-                                        (unsigned)(ix0 + ekx[e]) < (unsigned)g.W;
-                        e16[e] = in ? __ldg(x2 + base + eoff[e]) : (unsigned short)0;
-                    }
-                    uint4 v;
-                    v.x = e16[0] | ((uint32_t)e16[1] << 16);
-                    v.y = e16[2] | ((uint32_t)e16[3] << 16);
-                    v.z = e16[4] | ((uint32_t)e16[5] << 16);
-                    v.w = e16[6] | ((uint32_t)e16[7] << 16);
-                    ptx::st_shared_v4(((i & 1) ? dst_odd : dst_even) + (uint32_t)(i >> 1) * 1024u, v);
-                }
-                ptx::fence_proxy_async_smem();
-                ptx::mbar_arrive(ptx::smem_u32(&sh->full[s]));
             }
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));    // this stage no longer reads the row ring
+        } else {
+        int s = 0, j = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++j) {
+            const int r = j & (INFO_RING - 1);
+            if (!warp_wait_bar<100>(ptx::smem_u32(&sh->info_full[r]), (uint32_t)(j / INFO_RING) & 1u, abort_flag, a.dev_status)) break;
+            const int2* info = sh->rowinfo[r] + 16 * pw;
+            int pix[4], yx[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int2 ri = info[rq + 4 * i];
+                pix[i] = ri.x; yx[i] = ri.y;
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));    // the ring slot is in registers now
+
+            // window position of this lane's first K element of the stage
+            int ky, kx, ci;
+            {
+                const int k_first = c * 8;
+                const int tap = k_first / g.C_in;
+                ci = k_first - tap * g.C_in;
+                ky = tap / g.kw;
+                kx = tap - ky * g.kw;
+            }
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!warp_wait_bar<40>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
+                const uint32_t full = ptx::smem_u32(&sh->full[s]);
+                const uint32_t stage = smem_base + s * stage_bytes + (uint32_t)(16 * pw) * 128u;
+                if (MODE == GATHER_CPASYNC) {
+                    const bool kvalid = ky < g.kh;     // past K: the window is exhausted
+                    const int koff = ky * g.W + kx;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int row = rq + 4 * i;    // row & 7 == (rq + 4i) & 7
+                        const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
+                        const bool in = kvalid && (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
+                        const unsigned short* src = in ? x2 + ((long long)(pix[i] + koff) * g.C_in + ci) : x2;
+                        ptx::cp_async_16(stage + (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)), src, in ? 16u : 0u);
+                    }
+                    ptx::cp_async_mbar_arrive_noinc(full);
+                } else {
+                    int eoff[8], eky[8], ekx[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int k = kb * BK + c * 8 + e;
+                        const int tap = k / g.C_in, cie = k - tap * g.C_in;
+                        const int kye = tap / g.kw;
+                        eky[e] = (k < g.K) ? kye : (1 << 26);                 // past K: never in bounds
+                        ekx[e] = tap - kye * g.kw;
+                        eoff[e] = (kye * g.W + ekx[e]) * g.C_in + cie;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int row = rq + 4 * i;
+                        const int iy0 = yx[i] >> 16, ix0 = (int)(short)(yx[i] & 0xffff);
+                        unsigned short e16[8];
+                        const long long base = (long long)pix[i] * g.C_in;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const bool in = (unsigned)(iy0 + eky[e]) < (unsigned)g.H &&
+                                            (unsigned)(ix0 + ekx[e]) < (unsigned)g.W;
+                            e16[e] = in ? __ldg(x2 + base + eoff[e]) : (unsigned short)0;
+                        }
+                        uint4 v;
+                        v.x = e16[0] | ((uint32_t)e16[1] << 16);
+                        v.y = e16[2] | ((uint32_t)e16[3] << 16);
+                        v.z = e16[4] | ((uint32_t)e16[5] << 16);
+                        v.w = e16[6] | ((uint32_t)e16[7] << 16);
+                        ptx::st_shared_v4(stage + (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)), v);
+                    }
+                    ptx::fence_proxy_async_smem();
+                    ptx::mbar_arrive(full);
+                }
+                // advance the window position by 64 K elements
+                ci += BK;
+                while (ci >= g.C_in) {
+                    ci -= g.C_in;
+                    if (++kx == g.kw) { kx = 0; ++ky; }
+                }
+                if (++s == S) { s = 0; ph ^= 1u; }
+            }
         }
-        if (VEC) ptx::cp_async_wait<0>();          // nothing of this thread is in flight at exit
+        }
+        if (MODE == GATHER_CPASYNC) ptx::cp_async_wait<0>();      // nothing of this thread is in flight at exit
     }
 
     ptx::tc_fence_before_sync();
@@ -485,12 +575,28 @@ __global__ void repack_w_kernel(const unsigned short* __restrict__ w, unsigned s
 
 }  // namespace
 
-bool plan_fast(const ConvGeom& g, FastPlan* plan)
+bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, FastPlan* plan)
 {
     const int N = g.C_out;
-    const int n_tiles = (N + 255) / 256;
-    const int per = (N + n_tiles - 1) / n_tiles;
-    const int BN = ((per + 15) / 16) * 16;
+    const int KB = (g.K + BK - 1) / BK;
+    const long long m_tiles = (est_kept_rows + BM - 1) / BM > 0 ? (est_kept_rows + BM - 1) / BM : 1;
+    // Tile width: the widest tile (up to 256 columns) does the most work per gathered byte, but
+    // a layer with few kept rows then has fewer tiles than SMs.  Pick the width with the lowest
+    // estimated time = waves x k-blocks x max(copy issue time, MMA time) per k-block.
+    int best_BN = 0;
+    double best_cost = 0.0;
+    for (int n_tiles = (N + 255) / 256; ; n_tiles *= 2) {
+        const int per = (N + n_tiles - 1) / n_tiles;
+        const int BN = ((per + 15) / 16) * 16;
+        const int nt = (N + BN - 1) / BN;
+        const long long waves = (m_tiles * nt + num_sms - 1) / num_sms;
+        const double t_kb = 0.2 > BN * 0.0015 ? 0.2 : BN * 0.0015;          // microseconds, rough
+        const double cost = (double)waves * (KB * t_kb + 1.0);
+        if (best_BN == 0 || cost < best_cost * 0.98) { best_BN = BN; best_cost = cost; }
+        if (BN <= 64) break;
+    }
+    const int BN = best_BN;
+    const int n_tiles = (N + BN - 1) / BN;
     const int stage_bytes = A_STAGE_BYTES + BN * BK * 2;
     const int budget = 227 * 1024 - 1024 - (int)sizeof(Shared);
     int S = budget / stage_bytes;
@@ -502,13 +608,13 @@ bool plan_fast(const ConvGeom& g, FastPlan* plan)
     int smem = 1024 + S * stage_bytes + (int)sizeof(Shared);
     if (smem < 120 * 1024) smem = 120 * 1024;      // one block per SM: tensor memory is not shared out
     plan->smem_bytes = smem;
-    plan->vec = (g.C_in % 8 == 0) ? 1 : 0;
+    plan->vec = (g.C_in % 64 == 0) ? GATHER_TMA : (g.C_in % 8 == 0) ? GATHER_CPASYNC : GATHER_ELEM;
     plan->Kpad = ((g.K + BK - 1) / BK) * BK;
     return true;
 }
 
 cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorMap& tmap_w,
-                        const void* x, const float* bias, void* y, const uint8_t* mask,
+                        const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
                         int num_sms, cudaStream_t st)
 {
@@ -532,14 +638,16 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     long long tiles = ((long long)g.M + BM - 1) / BM * plan.n_tiles;
     int grid = (int)(tiles < num_sms ? tiles : num_sms);
     if (grid < 1) grid = 1;
-    auto kern = plan.vec ? masked_conv_sm100_kernel<true> : masked_conv_sm100_kernel<false>;
-    static int smem_set[2] = {0, 0};            // largest dynamic shared memory size enabled so far
+    auto kern = plan.vec == GATHER_TMA       ? masked_conv_sm100_kernel<GATHER_TMA>
+                : plan.vec == GATHER_CPASYNC ? masked_conv_sm100_kernel<GATHER_CPASYNC>
+                                             : masked_conv_sm100_kernel<GATHER_ELEM>;
+    static int smem_set[3] = {0, 0, 0};         // largest dynamic shared memory size enabled so far
     if (plan.smem_bytes > smem_set[plan.vec]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
         if (e != cudaSuccess) return e;
         smem_set[plan.vec] = plan.smem_bytes;
     }
-    kern<<<grid, NUM_THREADS, plan.smem_bytes, st>>>(tmap_w, g, a);
+    kern<<<grid, NUM_THREADS, plan.smem_bytes, st>>>(tmap_w, tmap_x, g, a);
     return cudaGetLastError();
 }
 
