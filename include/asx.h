@@ -164,6 +164,28 @@ asx_status asx_compact(const uint8_t* mask_dev, int64_t rows, int32_t* kept_dev,
  * buffer ran to completion (ASX_OK) or gave up in a bounded wait (ASX_ERR_TIMEOUT). */
 asx_status asx_compact_status(const void* scratch_dev, void* cuda_stream);
 
+/*
+ * Mask compaction without any allocation (the paper has no counterpart: this is a convenience
+ * of this library).  Same inputs, outputs and result as asx_compact, but the scan's scratch is
+ * a fixed array inside the library, so neither the caller nor the library allocates anything:
+ * no cudaMalloc, no cudaFree, no pooled allocator.  Meant for callers that cannot allocate where
+ * they stand: a latency-critical serving loop (cudaMalloc synchronises the device), code that
+ * runs after another framework took all device memory, a plug-in that only receives raw buffers.
+ *   rows : 0 <= rows <= ASX_COMPACT_STATIC_MAX_ROWS; more returns ASX_ERR_UNSUPPORTED and
+ *          launches nothing (use asx_compact with your own scratch instead).
+ *   mask_dev, kept_dev (room for `rows` int32), count_dev (one int32): device pointers as for
+ *          asx_compact.
+ * The array (about 32 KB) is part of the library image on every GPU that loads it.  The first
+ * call on each device looks up the array's device address; make that first call outside any
+ * stream capture.  All calls on a device share the one array: it is cleared on the stream at
+ * the start of each call, and two calls that may overlap on the GPU (different streams without
+ * an ordering between them) race on it and give undefined lists.  A bounded-wait timeout inside
+ * the kernel cannot be queried through this entry point.
+ */
+#define ASX_COMPACT_STATIC_MAX_ROWS (1 << 24)
+asx_status asx_compact_static(const uint8_t* mask_dev, int64_t rows, int32_t* kept_dev,
+                              int32_t* count_dev, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

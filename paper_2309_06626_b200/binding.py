@@ -15,8 +15,9 @@ ACT_RELU, RECOMPACT, IMPL_NAIVE = 1, 2, 4
 EXPORTS = (
     "asx_status_string", "asx_create_layer", "asx_set_mask", "asx_set_mask_random", "asx_recompact", "asx_run",
     "asx_get_kept", "asx_get_kept_host", "asx_get_mask", "asx_last_device_status", "asx_destroy",
-    "asx_compact_scratch_bytes", "asx_compact", "asx_compact_status",
+    "asx_compact_scratch_bytes", "asx_compact", "asx_compact_status", "asx_compact_static",
 )
+COMPACT_STATIC_MAX_ROWS = 1 << 24
 
 
 class AsxError(RuntimeError):
@@ -55,6 +56,7 @@ def lib():
         L.asx_compact_scratch_bytes.restype = i64
         L.asx_compact.argtypes = [vp, i64, vp, vp, vp, i64, vp]
         L.asx_compact_status.argtypes = [vp, vp]
+        L.asx_compact_static.argtypes = [vp, i64, vp, vp, vp]
         for name in EXPORTS:
             if name not in ("asx_status_string", "asx_compact_scratch_bytes"):
                 getattr(L, name).restype = ci

@@ -162,3 +162,57 @@ cudaError_t launch_compact(const uint8_t* mask, int64_t rows, int32_t* kept, int
 }
 
 }  // namespace asx
+
+// ---------------------------------------------------------------------------------------------
+// asx_compact_static: the same compaction for callers that must not allocate.
+//
+// The chained scan needs a little global scratch (a ticket, an error word and one 64-bit status
+// word per 4096-row tile).  Every other entry point takes that scratch from the caller or from
+// memory the layer allocated.  Some callers can do neither at the moment they need a kept-row
+// list: a serving loop that must not call cudaMalloc because it synchronises the whole device and
+// stalls every other stream; code running after a framework has claimed all device memory for
+// its own pool; a plug-in that only holds the raw buffers its host handed in.  For them the
+// scratch lives in the library image itself, in the array below: no allocation call of any
+// kind is made, at the price of a fixed upper size and of one array shared between all calls.
+namespace {
+
+constexpr long long STATIC_MAX_ROWS = ASX_COMPACT_STATIC_MAX_ROWS;
+constexpr size_t STATIC_SCRATCH_BYTES = 8 + 8 * (size_t)(STATIC_MAX_ROWS / asx::COMPACT_TILE);
+
+// Held by every GPU that loads the library until the process exits (about 32 KB).
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address the GPU
+// understands, so the device address is looked up once per device and remembered here.
+constexpr int MAX_DEVICES = 64;
+void* g_static_scratch_addr[MAX_DEVICES] = {nullptr};
+
+}  // namespace
+
+extern "C" asx_status asx_compact_static(const uint8_t* mask_dev, int64_t rows, int32_t* kept_dev,
+                                         int32_t* count_dev, void* cuda_stream)
+{
+    if (rows < 0 || count_dev == nullptr) return ASX_ERR_INVALID_ARG;
+    if (rows > 0 && (mask_dev == nullptr || kept_dev == nullptr)) return ASX_ERR_INVALID_ARG;
+    if (rows > STATIC_MAX_ROWS) return ASX_ERR_UNSUPPORTED;          // the built-in scratch is too small
+    if ((reinterpret_cast<uintptr_t>(kept_dev) & 3) || (reinterpret_cast<uintptr_t>(count_dev) & 3)) return ASX_ERR_ALIGN;
+    if ((size_t)asx::compact_scratch_bytes(rows) > STATIC_SCRATCH_BYTES) return ASX_ERR_UNSUPPORTED;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return ASX_ERR_CUDA;
+    if (dev < 0 || dev >= MAX_DEVICES) return ASX_ERR_UNSUPPORTED;
+    if (g_static_scratch_addr[dev] == nullptr) {
+        // first call on this device: resolve the array's device address (not a stream operation)
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return ASX_ERR_CUDA;
+        }
+        g_static_scratch_addr[dev] = p;
+    }
+    // launch_compact clears the ticket, the error word and the status words on the stream before
+    // the kernel runs, so whatever the previous call left in the array does not matter.
+    return asx::launch_compact(mask_dev, rows, kept_dev, count_dev, g_static_scratch_addr[dev],
+                               static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+               ? ASX_OK
+               : ASX_ERR_CUDA;
+}
