@@ -202,7 +202,7 @@ class DeviceLayer:
         self.bytes = wl.algorithmic_bytes(spec, self.mask)
         self.ptrs = (self.x.data_ptr(), spec.Nb, spec.H, spec.W, self.w.data_ptr(), self.b.data_ptr(),
                      self.y.data_ptr())
-        self.launches = 2 + (1 if spec.C_in % 8 else 0)      # compaction, main kernel, filter repack
+        self.launches = 2 + (2 if spec.C_in % 8 else 0)      # compaction, main kernel, channel padding of x and w
 
     def step(self, st, flags, layer=None):
         L = layer or self.layer

@@ -110,8 +110,9 @@ asx_status asx_recompact(asx_layer* layer, void* cuda_stream);
  *   y    : device, bf16 [Nb][Ho][Wo][C_out], Ho = (H + 2*pad - kh)/stride + 1 (Wo alike);
  *          16-byte aligned when C_out % 8 == 0, else 2-byte; must not overlap x.
  *   flags: OR of ASX_ACT_RELU, ASX_RECOMPACT, ASX_IMPL_NAIVE.
- * Asynchronous on `cuda_stream`; allocates only when a layer first needs a staging buffer
- * (C_in % 8 != 0) or when that buffer must grow.  Errors: ASX_ERR_NO_MASK, ASX_ERR_SHAPE when
+ * Asynchronous on `cuda_stream`; allocates only when C_in % 8 != 0: the layer then keeps copies of
+ * x and w with the channels zero-padded to a multiple of 8 (refreshed by a small kernel on every
+ * call), allocated on first use and when they must grow.  Errors: ASX_ERR_NO_MASK, ASX_ERR_SHAPE when
  * the mask length is neither Ho*Wo nor Nb*Ho*Wo, ASX_ERR_INVALID_ARG, ASX_ERR_ALIGN,
  * ASX_ERR_UNSUPPORTED when Nb*Ho*Wo or a tensor's element count reaches 2^31.
  */

@@ -23,9 +23,11 @@ struct asx_layer {
     int32_t* d_small = nullptr;        // [0] kept count, [1] status word
     bool has_mask = false;
     int64_t host_kept = -1;            // kept entries of the mask when it came from the host, else -1
-    // staging for filters whose K is not a multiple of 8
+    // staging copies with zero-padded channels, for C_in not a multiple of 8
     void* d_wpack = nullptr;
     size_t wpack_bytes = 0;
+    void* d_xpad = nullptr;
+    size_t xpad_bytes = 0;
     // tensor map cache
     CUtensorMap tmap;
     const void* tmap_ptr = nullptr;
@@ -282,28 +284,45 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     if (flags & ASX_IMPL_NAIVE)
         return from_cuda(launch_naive(g, x, w, bias, y, L->d_mask, L->d_kept, d_count, relu, st));
 
+    // Channel counts that are not a multiple of 8 are padded with zero channels in staging
+    // copies of x and w (a filter tap of a pixel is then a whole number of 16-byte chunks); the
+    // kernel runs on the padded geometry, the zero channels contribute nothing.
+    const void* xsrc = x;
+    const void* wsrc = w;
+    if (L->C_in % 8 != 0) {
+        const int Cp = (L->C_in + 7) / 8 * 8;
+        const int64_t pixels = (int64_t)Nb * H * W, taps = (int64_t)L->C_out * L->kh * L->kw;
+        if (pixels * Cp > lim) return ASX_ERR_UNSUPPORTED;
+        const size_t need_x = (size_t)pixels * Cp * 2, need_w = (size_t)taps * Cp * 2;
+        if (need_x > L->xpad_bytes || need_w > L->wpack_bytes) {
+            cudaStreamSynchronize(st);
+            if (need_x > L->xpad_bytes) {
+                cudaFree(L->d_xpad);
+                L->d_xpad = nullptr; L->xpad_bytes = 0;
+                if (cudaMalloc(&L->d_xpad, need_x) != cudaSuccess) return ASX_ERR_OOM;
+                L->xpad_bytes = need_x;
+            }
+            if (need_w > L->wpack_bytes) {
+                cudaFree(L->d_wpack);
+                L->d_wpack = nullptr; L->wpack_bytes = 0;
+                if (cudaMalloc(&L->d_wpack, need_w) != cudaSuccess) return ASX_ERR_OOM;
+                L->wpack_bytes = need_w;
+            }
+            L->tmap_ptr = nullptr;
+        }
+        cudaError_t e = launch_pad_channels(x, L->d_xpad, pixels, L->C_in, Cp, st);
+        if (e == cudaSuccess) e = launch_pad_channels(w, L->d_wpack, taps, L->C_in, Cp, st);
+        if (e != cudaSuccess) return from_cuda(e);
+        xsrc = L->d_xpad;
+        wsrc = L->d_wpack;
+        g.C_in = Cp;
+        g.K = L->kh * L->kw * Cp;
+    }
     FastPlan plan;
     long long est_rows = M;                                       // unknown on the host: assume every row kept
     if (L->host_kept >= 0) est_rows = (L->rows == P) ? L->host_kept * Nb : L->host_kept;
     if (!plan_fast(g, L->num_sms, est_rows, &plan)) return ASX_ERR_UNSUPPORTED;
-    const void* wsrc = w;
-    int Kw = g.K;
-    if (!plan.vec) {
-        // filters whose rows are not a multiple of 16 bytes are staged into a padded copy
-        Kw = (g.K + 7) / 8 * 8;
-        const size_t need = (size_t)L->C_out * Kw * 2;
-        if (need > L->wpack_bytes) {
-            cudaStreamSynchronize(st);
-            cudaFree(L->d_wpack);
-            L->d_wpack = nullptr; L->wpack_bytes = 0;
-            if (cudaMalloc(&L->d_wpack, need) != cudaSuccess) return ASX_ERR_OOM;
-            L->wpack_bytes = need;
-            L->tmap_ptr = nullptr;
-        }
-        cudaError_t e = launch_repack_w(w, L->d_wpack, L->C_out, g.K, Kw, st);
-        if (e != cudaSuccess) return from_cuda(e);
-        wsrc = L->d_wpack;
-    }
+    const int Kw = g.K;
     if (L->tmap_ptr != wsrc || L->tmap_BN != plan.BN || L->tmap_Kw != Kw) {
         EncodeTiledFn enc = encode_tiled_fn();
         if (enc == nullptr) return ASX_ERR_CUDA;
@@ -319,21 +338,21 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     }
     if (plan.vec == 2) {
         const int64_t pixels = (int64_t)Nb * H * W;
-        if (L->tmapx_ptr != x || L->tmapx_pixels != pixels) {
+        if (L->tmapx_ptr != xsrc || L->tmapx_pixels != pixels) {
             EncodeTiledFn enc = encode_tiled_fn();
             if (enc == nullptr) return ASX_ERR_CUDA;
-            const cuuint64_t dims[2] = {(cuuint64_t)L->C_in, (cuuint64_t)pixels};
-            const cuuint64_t strides[1] = {(cuuint64_t)L->C_in * 2};
+            const cuuint64_t dims[2] = {(cuuint64_t)g.C_in, (cuuint64_t)pixels};
+            const cuuint64_t strides[1] = {(cuuint64_t)g.C_in * 2};
             const cuuint32_t box[2] = {64u, 1u};
             const cuuint32_t estr[2] = {1u, 1u};
-            const CUresult r = enc(&L->tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims,
+            const CUresult r = enc(&L->tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(xsrc), dims,
                                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return ASX_ERR_CUDA;
-            L->tmapx_ptr = x; L->tmapx_pixels = pixels;
+            L->tmapx_ptr = xsrc; L->tmapx_pixels = pixels;
         }
     }
-    return from_cuda(launch_fast(g, plan, L->tmap, plan.vec == 2 ? L->tmap_x : L->tmap, x, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
+    return from_cuda(launch_fast(g, plan, L->tmap, plan.vec == 2 ? L->tmap_x : L->tmap, xsrc, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
                                  L->num_sms, st));
 }
 
@@ -393,7 +412,7 @@ asx_status asx_destroy(asx_layer* L)
     if (L->device >= 0) {
         cudaStreamSynchronize(L->last_stream);
         cudaFree(L->d_mask); cudaFree(L->d_kept); cudaFree(L->d_scratch);
-        cudaFree(L->d_small); cudaFree(L->d_wpack);
+        cudaFree(L->d_small); cudaFree(L->d_wpack); cudaFree(L->d_xpad);
     }
     delete L;
     return ASX_OK;

@@ -19,7 +19,28 @@ struct ConvGeom {
 // Device status word values (bit flags), reported as ASX_ERR_TIMEOUT.
 enum : int { DEV_OK = 0, DEV_TIMEOUT_SCAN = 1, DEV_TIMEOUT_PIPE = 2, DEV_BAD_INDEX = 4 };
 
+// Launch with the programmatic-stream-serialization attribute: the kernel may begin while its
+// predecessor in the stream is still running and must execute griddepcontrol.wait before it
+// touches anything an earlier kernel produced (and before it writes anything one may still read).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- S1: mask compaction (compact.cu)
+constexpr int COMPACT_SMALL_MAX_ROWS = 1024 * 16;   // one block handles masks up to this size
 constexpr int COMPACT_THREADS = 256;
 constexpr int COMPACT_PER_THREAD = 16;
 constexpr int COMPACT_TILE = COMPACT_THREADS * COMPACT_PER_THREAD;
@@ -38,8 +59,7 @@ struct FastPlan {
     int n_tiles;      // ceil(C_out / BN)
     int stages;
     int smem_bytes;
-    int vec;          // gather mode: 0 element loads (any C_in), 1 cp.async 16 B (C_in % 8 == 0),
-                      // 2 TMA row gather (C_in % 64 == 0)
+    int vec;          // gather mode: 1 cp.async 16 B (C_in % 8 == 0), 2 TMA row gather (C_in % 64 == 0)
     int Kpad;         // K rounded up to 64
 };
 bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, FastPlan* plan);
@@ -47,7 +67,7 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
                         const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
                         int num_sms, cudaStream_t st);
-// repack w[C_out][K] into wp[C_out][Kw] (zero padded), for K not a multiple of 8
-cudaError_t launch_repack_w(const void* w, void* wp, int C_out, int K, int Kw, cudaStream_t st);
+// src[rows][C] -> dst[rows][Cp] with zero channels added (Cp a multiple of 8)
+cudaError_t launch_pad_channels(const void* src, void* dst, long long rows, int C, int Cp, cudaStream_t st);
 
 }  // namespace asx

@@ -10,6 +10,7 @@
 // ticket so that every predecessor of a running tile has already started; the look-back
 // wait is bounded and reports through the error word instead of spinning for ever.
 #include "asx_internal.h"
+#include "ptx_sm100.cuh"
 
 namespace asx {
 
@@ -41,6 +42,8 @@ compact_kernel(const uint8_t* __restrict__ mask, long long rows, int32_t* __rest
     __shared__ int s_exclusive;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();          // the list being rebuilt may still be read by an earlier kernel
     if (tid == 0) s_tile = (int)atomicAdd(&hdr->ticket, 1u);
     __syncthreads();
     const int tile = s_tile;
@@ -136,6 +139,59 @@ compact_kernel(const uint8_t* __restrict__ mask, long long rows, int32_t* __rest
     if (tile == num_tiles - 1 && tid == 0) *count = exclusive + tile_total;
 }
 
+// Masks of up to 16 384 rows (every per-layer mask of a classification network) need no chained
+// scan: one block of 1024 threads, 16 mask bytes per thread, a shuffle scan within and across
+// the warps, and each thread writes its own indices.  No ticket, no status words, no clearing.
+__global__ void __launch_bounds__(1024)
+compact_small_kernel(const uint8_t* __restrict__ mask, int rows, int32_t* __restrict__ kept,
+                     int32_t* __restrict__ count, ScratchHeader* hdr)
+{
+    __shared__ int s_warp_total[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
+    const int first = tid * COMPACT_PER_THREAD;
+    unsigned flags = 0;
+    const bool aligned = (reinterpret_cast<uintptr_t>(mask) & 15) == 0;
+    if (aligned && first + COMPACT_PER_THREAD <= rows) {
+        const uint4 v = *reinterpret_cast<const uint4*>(mask + first);
+        flags = nonzero_bytes4(v.x) | (nonzero_bytes4(v.y) << 4) | (nonzero_bytes4(v.z) << 8) |
+                (nonzero_bytes4(v.w) << 12);
+    } else {
+        for (int j = 0; j < COMPACT_PER_THREAD; ++j)
+            if (first + j < rows && mask[first + j] != 0) flags |= 1u << j;
+    }
+    const int mine = __popc(flags);
+    int incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += t;
+    }
+    if (lane == 31) s_warp_total[warp] = incl;
+    __syncthreads();
+    // every warp scans the 32 warp totals itself: lane i holds the total of warp i
+    int wt = s_warp_total[lane], winc = wt;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, winc, d);
+        if (lane >= d) winc += t;
+    }
+    const int warp_prefix = __shfl_sync(0xffffffffu, winc - wt, warp);
+    const int total = __shfl_sync(0xffffffffu, winc, 31);
+    int at = warp_prefix + incl - mine;
+    unsigned f = flags;
+    while (f) {
+        const int j = __ffs(f) - 1;
+        f &= f - 1;
+        kept[at++] = first + j;
+    }
+    if (tid == 0) {
+        *count = total;
+        if (hdr != nullptr) { hdr->ticket = 0; hdr->error = 0; }     // a status query must find a clean word
+    }
+}
+
 }  // namespace
 
 static int tiles_for(int64_t rows)
@@ -152,13 +208,15 @@ int64_t compact_scratch_bytes(int64_t rows)
 cudaError_t launch_compact(const uint8_t* mask, int64_t rows, int32_t* kept, int32_t* count,
                            void* scratch, cudaStream_t st)
 {
+    auto* hdr = static_cast<ScratchHeader*>(scratch);
+    if (rows <= COMPACT_SMALL_MAX_ROWS)
+        return launch_pdl(compact_small_kernel, dim3(1), dim3(1024), 0, st, mask, (int)rows, kept, count, hdr);
     const int tiles = tiles_for(rows);
     cudaError_t e = cudaMemsetAsync(scratch, 0, (size_t)compact_scratch_bytes(rows), st);
     if (e != cudaSuccess) return e;
-    auto* hdr = static_cast<ScratchHeader*>(scratch);
-    auto* status = reinterpret_cast<unsigned long long*>(hdr + 1);
-    compact_kernel<<<tiles, COMPACT_THREADS, 0, st>>>(mask, (long long)rows, kept, count, hdr, status, tiles);
-    return cudaGetLastError();
+    auto* status = reinterpret_cast<volatile unsigned long long*>(hdr + 1);
+    return launch_pdl(compact_kernel, dim3(tiles), dim3(COMPACT_THREADS), 0, st, mask, (long long)rows, kept, count,
+                      hdr, status, tiles);
 }
 
 }  // namespace asx
@@ -209,8 +267,8 @@ extern "C" asx_status asx_compact_static(const uint8_t* mask_dev, int64_t rows, 
         }
         g_static_scratch_addr[dev] = p;
     }
-    // launch_compact clears the ticket, the error word and the status words on the stream before
-    // the kernel runs, so whatever the previous call left in the array does not matter.
+    // launch_compact clears (or, for small masks, never uses) the ticket, the error word and the
+    // status words on the stream, so whatever the previous call left in the array does not matter.
     return asx::launch_compact(mask_dev, rows, kept_dev, count_dev, g_static_scratch_addr[dev],
                                static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
                ? ASX_OK

@@ -115,7 +115,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-enum : int { GATHER_ELEM = 0, GATHER_CPASYNC = 1, GATHER_TMA = 2 };
+enum : int { GATHER_CPASYNC = 1, GATHER_TMA = 2 };
 
 template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -125,23 +125,10 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     extern __shared__ uint8_t smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    const int cnt = *a.count;
-    const int Mk = (g.rows == g.P) ? g.Nb * cnt : cnt;
+    // Let the next kernel of the stream start its own prologue; everything up to the dependency
+    // wait below touches only this block's shared and tensor memory.
+    ptx::grid_launch_dependents();
     const int N = g.C_out;
-
-    if (Mk <= 0) {
-        // every position dropped: the whole output is zeros (Algorithm 2, mask == 0 branch)
-        const long long total = (long long)g.M * N;
-        const long long t = blockIdx.x * (long long)NUM_THREADS + tid, step = (long long)gridDim.x * NUM_THREADS;
-        if (a.vec_out) {
-            uint4* y16 = reinterpret_cast<uint4*>(a.y);
-            for (long long i = t; i < total / 8; i += step) y16[i] = make_uint4(0, 0, 0, 0);
-        } else {
-            unsigned short* y2 = reinterpret_cast<unsigned short*>(a.y);
-            for (long long i = t; i < total; i += step) y2[i] = 0;
-        }
-        return;
-    }
 
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     const int BN = a.BN, S = a.stages;
@@ -150,8 +137,6 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     volatile int* abort_flag = &sh->abort;
 
     const int KB = (g.K + BK - 1) / BK;
-    const int m_tiles = (Mk + BM - 1) / BM;
-    const int total_tiles = m_tiles * a.n_tiles;
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
@@ -183,6 +168,16 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
+
+    // From here on the kernel reads what earlier kernels wrote (the kept-row list and its count,
+    // the input) and writes the output, so it waits for them to have finished.
+    ptx::grid_dependency_wait();
+    const int cnt = *a.count;
+    const int Mk = (g.rows == g.P) ? g.Nb * cnt : cnt;
+    // With every position dropped there are no tiles; the zero warps then write the whole output
+    // (Algorithm 2, mask == 0 branch).
+    const int m_tiles = (Mk + BM - 1) / BM;
+    const int total_tiles = m_tiles * a.n_tiles;
 
     if (warp == WARP_TMA) {
         // ------------------------------------------------------------------ filter slabs by TMA
@@ -495,7 +490,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                 if (!warp_wait_bar<40>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
                 const uint32_t full = ptx::smem_u32(&sh->full[s]);
                 const uint32_t stage = smem_base + s * stage_bytes + (uint32_t)(16 * pw) * 128u;
-                if (MODE == GATHER_CPASYNC) {
+                {
                     const bool kvalid = ky < g.kh;     // past K: the window is exhausted
                     const int koff = ky * g.W + kx;
 #pragma unroll
@@ -507,38 +502,6 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                         ptx::cp_async_16(stage + (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)), src, in ? 16u : 0u);
                     }
                     ptx::cp_async_mbar_arrive_noinc(full);
-                } else {
-                    int eoff[8], eky[8], ekx[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const int k = kb * BK + c * 8 + e;
-                        const int tap = k / g.C_in, cie = k - tap * g.C_in;
-                        const int kye = tap / g.kw;
-                        eky[e] = (k < g.K) ? kye : (1 << 26);                 // past K: never in bounds
-                        ekx[e] = tap - kye * g.kw;
-                        eoff[e] = (kye * g.W + ekx[e]) * g.C_in + cie;
-                    }
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int row = rq + 4 * i;
-                        const int iy0 = yx[i] >> 16, ix0 = (int)(short)(yx[i] & 0xffff);
-                        unsigned short e16[8];
-                        const long long base = (long long)pix[i] * g.C_in;
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            const bool in = (unsigned)(iy0 + eky[e]) < (unsigned)g.H &&
-                                            (unsigned)(ix0 + ekx[e]) < (unsigned)g.W;
-                            e16[e] = in ? __ldg(x2 + base + eoff[e]) : (unsigned short)0;
-                        }
-                        uint4 v;
-                        v.x = e16[0] | ((uint32_t)e16[1] << 16);
-                        v.y = e16[2] | ((uint32_t)e16[3] << 16);
-                        v.z = e16[4] | ((uint32_t)e16[5] << 16);
-                        v.w = e16[6] | ((uint32_t)e16[7] << 16);
-                        ptx::st_shared_v4(stage + (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)), v);
-                    }
-                    ptx::fence_proxy_async_smem();
-                    ptx::mbar_arrive(full);
                 }
                 // advance the window position by 64 K elements
                 ci += BK;
@@ -562,14 +525,29 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     }
 }
 
-__global__ void repack_w_kernel(const unsigned short* __restrict__ w, unsigned short* __restrict__ wp,
-                                int C_out, int K, int Kw)
+// Channel padding: src[rows][C] -> dst[rows][Cp], Cp a multiple of 8, zeros in the added channels.
+// Used for inputs and filters whose channel count is not a multiple of 8, so that every filter
+// tap of a pixel is a whole number of 16-byte chunks.  One thread per 16-byte chunk of dst.
+__global__ void pad_channels_kernel(const unsigned short* __restrict__ src, uint4* __restrict__ dst,
+                                    long long rows, int C, int Cp)
 {
-    const long long total = (long long)C_out * Kw;
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
+    const int cpr = Cp >> 3;
+    const long long total = rows * cpr;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
-        const int co = (int)(i / Kw), k = (int)(i - (long long)co * Kw);
-        wp[i] = (k < K) ? w[(long long)co * K + k] : (unsigned short)0;
+        const long long row = i / cpr;
+        const int c0 = (int)(i - row * cpr) * 8;
+        unsigned short e[8];
+#pragma unroll
+        for (int q2 = 0; q2 < 8; ++q2) e[q2] = (c0 + q2 < C) ? src[row * C + c0 + q2] : (unsigned short)0;
+        uint4 v;
+        v.x = e[0] | ((uint32_t)e[1] << 16);
+        v.y = e[2] | ((uint32_t)e[3] << 16);
+        v.z = e[4] | ((uint32_t)e[5] << 16);
+        v.w = e[6] | ((uint32_t)e[7] << 16);
+        dst[i] = v;
     }
 }
 
@@ -608,7 +586,8 @@ bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, FastPlan
     int smem = 1024 + S * stage_bytes + (int)sizeof(Shared);
     if (smem < 120 * 1024) smem = 120 * 1024;      // one block per SM: tensor memory is not shared out
     plan->smem_bytes = smem;
-    plan->vec = (g.C_in % 64 == 0) ? GATHER_TMA : (g.C_in % 8 == 0) ? GATHER_CPASYNC : GATHER_ELEM;
+    if (g.C_in % 8 != 0) return false;            // the caller pads the channels first
+    plan->vec = (g.C_in % 64 == 0) ? GATHER_TMA : GATHER_CPASYNC;
     plan->Kpad = ((g.K + BK - 1) / BK) * BK;
     return true;
 }
@@ -638,27 +617,23 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     long long tiles = ((long long)g.M + BM - 1) / BM * plan.n_tiles;
     int grid = (int)(tiles < num_sms ? tiles : num_sms);
     if (grid < 1) grid = 1;
-    auto kern = plan.vec == GATHER_TMA       ? masked_conv_sm100_kernel<GATHER_TMA>
-                : plan.vec == GATHER_CPASYNC ? masked_conv_sm100_kernel<GATHER_CPASYNC>
-                                             : masked_conv_sm100_kernel<GATHER_ELEM>;
+    auto kern = plan.vec == GATHER_TMA ? masked_conv_sm100_kernel<GATHER_TMA> : masked_conv_sm100_kernel<GATHER_CPASYNC>;
     static int smem_set[3] = {0, 0, 0};         // largest dynamic shared memory size enabled so far
     if (plan.smem_bytes > smem_set[plan.vec]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
         if (e != cudaSuccess) return e;
         smem_set[plan.vec] = plan.smem_bytes;
     }
-    kern<<<grid, NUM_THREADS, plan.smem_bytes, st>>>(tmap_w, tmap_x, g, a);
-    return cudaGetLastError();
+    return launch_pdl(kern, dim3(grid), dim3(NUM_THREADS), (size_t)plan.smem_bytes, st, tmap_w, tmap_x, g, a);
 }
 
-cudaError_t launch_repack_w(const void* w, void* wp, int C_out, int K, int Kw, cudaStream_t st)
+cudaError_t launch_pad_channels(const void* src, void* dst, long long rows, int C, int Cp, cudaStream_t st)
 {
-    const long long total = (long long)C_out * Kw;
-    int blocks = (int)((total + 255) / 256 < 1024 ? (total + 255) / 256 : 1024);
+    const long long total = rows * (Cp / 8);
+    int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     if (blocks < 1) blocks = 1;
-    repack_w_kernel<<<blocks, 256, 0, st>>>(static_cast<const unsigned short*>(w),
-                                            static_cast<unsigned short*>(wp), C_out, K, Kw);
-    return cudaGetLastError();
+    return launch_pdl(pad_channels_kernel, dim3(blocks), dim3(256), 0, st, static_cast<const unsigned short*>(src),
+                      static_cast<uint4*>(dst), rows, C, Cp);
 }
 
 }  // namespace asx

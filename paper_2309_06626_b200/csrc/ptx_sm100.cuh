@@ -11,6 +11,18 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p)
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// Programmatic dependent launch: let the next kernel in the stream start its prologue now, and
+// wait until every kernel this one depends on has finished and its writes are visible.  Both are
+// no-ops for a kernel that was launched without the programmatic-serialization attribute.
+__device__ __forceinline__ void grid_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // One lane of a converged warp (elect.sync); the choice is the same on every call.
 __device__ __forceinline__ bool elect_one()
 {
