@@ -217,6 +217,7 @@ def run_ours(args):
     import torch.distributed as dist
     import paper_2309_06626_b200 as asx
     from paper_2309_06626_b200 import build as asx_build
+    from paper_2309_06626_b200.dist_util import max_over_ranks, whole_job_rate
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -241,13 +242,13 @@ def run_ours(args):
         specs = [s for s in specs if any(s.name.startswith(p) for p in args.only.split(","))]
         if not specs:
             raise SystemExit(f"--only {args.only}: no such layer")
-    layers = [DeviceLayer(s, torch, asx) for s in specs]
+    layers = [DeviceLayer(s, torch, asx, dense_twin=(args.config != 5)) for s in specs]
     torch.cuda.synchronize()
     footprint = sum(L.x.numel() * 2 + L.y.numel() * 2 + L.w.numel() * 2 for L in layers)
 
     def one_step(dense=False):
         for L in layers:
-            L.step(st, RELU, L.dense if dense else None)
+            L.step(st, RELU, L.dense if (dense and L.dense is not None) else None)
 
     def barrier():
         if world > 1:
@@ -308,11 +309,7 @@ def run_ours(args):
             row.append((a, b))
         probe_events.append(row)
     barrier()
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(e0.elapsed_time(e1), device="cuda")
     ms_step = ms_total / K
     for L in layers:
         if L.layer.device_status() != 0:
@@ -320,7 +317,7 @@ def run_ours(args):
 
     flops_step = sum(L.flops for L in layers)
     dense_flops_step = sum(L.flops_dense for L in layers)
-    value = world * flops_step / (ms_step * 1e-3) / 1e12
+    value = whole_job_rate(flops_step, ms_step, world) / 1e12
 
     # main-kernel durations (dominant kernel), per layer, averaged over the probed steps
     per_layer_ms = [statistics.mean(row[i][0].elapsed_time(row[i][1]) for row in probe_events)
@@ -380,11 +377,8 @@ def run_ours(args):
         e2e_step()
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - tw0) * 1e3 / Ke
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_val = world * flops_step / (e2e_ms * 1e-3) / 1e12
+    e2e_ms = max_over_ranks(e2e_ms, device="cuda")
+    e2e_val = whole_job_rate(flops_step, e2e_ms, world) / 1e12
     t_gpu_end = time.time()
 
     if rank != 0:
@@ -398,6 +392,49 @@ def run_ours(args):
         clocks = clocks_all
     cpu = None if args.no_cpu_baseline else cpu_baseline(args.config)
 
+    # ---- S1 alone on a mask large enough to be HBM-bound (the per-layer masks are a few KB)
+    s1 = None
+    if not args.no_s1:
+        rows = 1 << 27
+        gen = torch.Generator(device="cuda"); gen.manual_seed(wl.BASE_SEED)
+        big = (torch.rand(rows, device="cuda", generator=gen) < 0.5).to(torch.uint8)
+        kept_big = torch.empty(rows, dtype=torch.int32, device="cuda")
+        cnt_big = torch.empty(1, dtype=torch.int32, device="cuda")
+        nb = asx.lib().asx_compact_scratch_bytes(rows)
+        scr = torch.empty((nb + 7) // 8, dtype=torch.int64, device="cuda")
+
+        def s1_call():
+            rc = asx.lib().asx_compact(big.data_ptr(), rows, kept_big.data_ptr(), cnt_big.data_ptr(),
+                                       scr.data_ptr(), scr.numel() * 8, st)
+            if rc:
+                raise RuntimeError(f"asx_compact failed with status {rc}")
+        for _ in range(3):
+            s1_call()
+        torch.cuda.synchronize()
+        if asx.lib().asx_compact_status(scr.data_ptr(), st) != 0:
+            raise RuntimeError("compaction reported a bounded-wait timeout")
+        s0, s1e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(st_obj)
+        for _ in range(10):
+            s1_call()
+        s1e.record(st_obj)
+        torch.cuda.synchronize()
+        ms = s0.elapsed_time(s1e) / 10
+        kept_n = int(cnt_big.item())
+        gbs = (rows + 4 * kept_n) / (ms * 1e-3) / 1e9
+        s1 = {"rows": rows, "kept": kept_n, "ms": ms, "gbs": gbs, "bytes": "rows + 4*kept (mask read, list written)",
+              "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "peak_gbs": peaks["hbm_gbs"]}
+        del big, kept_big, scr
+
+    sweep = None
+    if args.config == 5:
+        base = {L.spec.block: per_layer_ms[i] for i, L in enumerate(layers) if L.spec.sparsity_pct == 0}
+        sweep = [{"sparsity_pct": L.spec.sparsity_pct, "block": L.spec.block, "ms": per_layer_ms[i],
+                  "tflops": L.flops / (per_layer_ms[i] * 1e-3) / 1e12,
+                  "speedup_vs_sparsity0": base[L.spec.block] / per_layer_ms[i],
+                  "ideal_speedup": layers[i].spec.M / max(1, L.kept_rows)}
+                 for i, L in enumerate(layers)]
+
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": K,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -410,7 +447,7 @@ def run_ours(args):
                            + ("" if graph is None else "; one step = one CUDA-graph replay"),
                    "mask": "one mask per layer shared by the batch"},
         "dense_equivalent_tflops": world * dense_flops_step / (ms_step * 1e-3) / 1e12,
-        "speedup_vs_sparsity0": ms_dense / ms_step,
+        "speedup_vs_sparsity0": (ms_dense / ms_step) if args.config != 5 else None,
         "ms_per_step_sparsity0": ms_dense,
         "speedup_vs_cudnn_dense": (cudnn_ms / ms_step) if cudnn_ms else None,
         "cudnn_dense_ms_per_step": cudnn_ms,
@@ -425,6 +462,8 @@ def run_ours(args):
                      "frac_of_layer_roofs": roof_ms / kern_ms,
                      "layer_roofs_ms_per_step": roof_ms},
         "cpu_baseline": cpu,
+        "s1_compaction": s1,
+        "sweep": sweep,
         "per_layer": [{"name": L.spec.name, "M": L.spec.M, "K": L.spec.K, "N": L.spec.N, "kept_rows": L.kept_rows,
                        "ms": per_layer_ms[i], "tflops": L.flops / (per_layer_ms[i] * 1e-3) / 1e12,
                        "gbs": L.bytes / (per_layer_ms[i] * 1e-3) / 1e9}
@@ -441,7 +480,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4])
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--no-s1", action="store_true", help="skip the stand-alone compaction bandwidth leg")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cudnn", action="store_true")

@@ -36,7 +36,7 @@ constexpr int MIN_STAGES = 4;
 constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_EPI0 = 2, WARP_PROD0 = 6;
 constexpr int NUM_PROD_WARPS = 8, NUM_EPI_WARPS = 4;
 constexpr int INFO_RING = 8;            // tiles whose row coordinates are kept in shared memory (power of two)
-constexpr int WARP_ZERO0 = WARP_PROD0 + NUM_PROD_WARPS, NUM_ZERO_WARPS = 2;
+constexpr int WARP_ZERO0 = WARP_PROD0 + NUM_PROD_WARPS, NUM_ZERO_WARPS = 4;
 constexpr int WARP_INFO = WARP_ZERO0 + NUM_ZERO_WARPS;
 constexpr int NUM_THREADS = 32 * (WARP_INFO + 1);
 constexpr long long WAIT_CYCLE_LIMIT = 4000000000ll;   // about two seconds
@@ -352,54 +352,54 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     } else if (warp >= WARP_ZERO0) {   // (the row-coordinate warp was handled above)
         // ------------------------------------------------------------------ zeros for dropped rows
         // Algorithm 2's post-processing writes zeros wherever the mask is 0.  These warps stream
-        // over this block's share of the output rows, independent of the tile loop: a warp reads
-        // 32 mask bytes (one per lane), a ballot gives the dropped rows, and the lanes write those
-        // rows together.  Kept rows are written by the epilogue, so each element is written once.
+        // over this block's share of the output rows, independent of the tile loop.  Kept rows
+        // are written by the epilogue, so each element is written exactly once.
+        // Fast path (16-byte stores, chunks per row dividing the thread count): every thread keeps
+        // one 16-byte column of the row and walks down the rows with a constant stride, so a warp
+        // writes whole consecutive rows; four mask bytes are fetched before the four stores they
+        // guard, and nothing in the loop divides.
         unsigned short* y2 = reinterpret_cast<unsigned short*>(a.y);
         const long long lo = (long long)g.M * blockIdx.x / gridDim.x;
         const long long hi = (long long)g.M * (blockIdx.x + 1) / gridDim.x;
-        const int zw = warp - WARP_ZERO0;
-        const int cpr = N >> 3;                                   // 16-byte chunks per row (vector path)
-        const int rows_per_pass = (a.vec_out && cpr < 32) ? 32 / cpr : 1;
-        const int sub = (a.vec_out && cpr < 32) ? lane / cpr : 0;
-        const int cc = (a.vec_out && cpr < 32) ? lane - sub * cpr : lane;
-        auto is_dropped = [&](long long row) -> bool {
-            if (row >= hi) return false;
-            const int r = (int)row;
-            return __ldg(a.mask + ((g.rows == g.P) ? r % g.P : r)) == 0;
-        };
-        long long base = lo + zw * 32;
-        bool d0 = is_dropped(base + lane);
-        bool d1 = is_dropped(base + NUM_ZERO_WARPS * 32 + lane);
-        while (base < hi) {
-            const unsigned dm = __ballot_sync(0xffffffffu, d0);
-            const long long cur = base;
-            base += NUM_ZERO_WARPS * 32;
-            d0 = d1;
-            d1 = is_dropped(base + NUM_ZERO_WARPS * 32 + lane);   // two groups ahead
-            unsigned rest = dm;
-            if (a.vec_out && cpr < 32) {
-                while (rest) {
-                    int mine = -1;                                  // the sub-th dropped row of this pass
-                    for (int q2 = 0; q2 < rows_per_pass && rest; ++q2) {
-                        const int bit = __ffs(rest) - 1;
-                        rest &= rest - 1;
-                        if (q2 == sub) mine = bit;
-                    }
-                    if (mine >= 0 && sub < rows_per_pass)
-                        *reinterpret_cast<uint4*>(y2 + (cur + mine) * N + cc * 8) = make_uint4(0, 0, 0, 0);
+        constexpr int ZT = NUM_ZERO_WARPS * 32;
+        const int zt = (warp - WARP_ZERO0) * 32 + lane;
+        const int cpr = N >> 3;                                   // 16-byte chunks per row
+        const bool shared_mask = (g.rows == g.P);
+        if (a.vec_out && cpr <= ZT && ZT % cpr == 0) {
+            const int rpp = ZT / cpr;                             // rows covered by one pass of all threads
+            const int sub = zt / cpr, cc = zt - sub * cpr;
+            long long row = lo + sub;
+            int p = shared_mask ? (int)(row % g.P) : 0;           // mask index of `row`, kept incrementally
+            const int pstep = rpp % g.P;
+            uint4* dst = reinterpret_cast<uint4*>(y2 + row * N + cc * 8);
+            const long long dstep = (long long)rpp * cpr;         // in 16-byte units
+            while (row < hi) {
+                bool drop[4];
+                int pk = p;
+#pragma unroll
+                for (int k2 = 0; k2 < 4; ++k2) {
+                    const long long rk = row + (long long)k2 * rpp;
+                    drop[k2] = (rk < hi) && __ldg(a.mask + (shared_mask ? (long long)pk : rk)) == 0;
+                    pk += pstep;
+                    if (pk >= g.P) pk -= g.P;
                 }
-            } else if (a.vec_out) {
-                while (rest) {
-                    const long long row = cur + __ffs(rest) - 1;
-                    rest &= rest - 1;
+#pragma unroll
+                for (int k2 = 0; k2 < 4; ++k2)
+                    if (drop[k2]) dst[k2 * dstep] = make_uint4(0, 0, 0, 0);
+                p = pk;
+                row += 4LL * rpp;
+                dst += 4 * dstep;
+            }
+        } else {
+            // general path: one warp per dropped row
+            const int zw = warp - WARP_ZERO0;
+            for (long long row = lo + zw; row < hi; row += NUM_ZERO_WARPS) {
+                const long long pm = shared_mask ? row % g.P : row;
+                if (__ldg(a.mask + pm) != 0) continue;
+                if (a.vec_out) {
                     for (int c1 = lane; c1 < cpr; c1 += 32)
                         *reinterpret_cast<uint4*>(y2 + row * N + c1 * 8) = make_uint4(0, 0, 0, 0);
-                }
-            } else {
-                while (rest) {
-                    const long long row = cur + __ffs(rest) - 1;
-                    rest &= rest - 1;
+                } else {
                     for (int c1 = lane; c1 < N; c1 += 32) y2[row * N + c1] = 0;
                 }
             }
