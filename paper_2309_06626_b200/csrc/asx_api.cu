@@ -249,6 +249,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     ConvGeom g;
     g.Nb = Nb; g.H = H; g.W = W; g.C_in = L->C_in; g.C_out = L->C_out;
     g.kh = L->kh; g.kw = L->kw; g.stride = L->stride; g.pad = L->pad;
+    g.stride_w = L->stride; g.pad_w = L->pad;
     g.Ho = (H + 2 * L->pad - L->kh) / L->stride + 1;
     g.Wo = (W + 2 * L->pad - L->kw) / L->stride + 1;
     g.K = L->kh * L->kw * L->C_in;
@@ -290,10 +291,19 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     const void* xsrc = x;
     const void* wsrc = w;
     if (L->C_in % 8 != 0) {
-        const int Cp = (L->C_in + 7) / 8 * 8;
-        const int64_t pixels = (int64_t)Nb * H * W, taps = (int64_t)L->C_out * L->kh * L->kw;
+        // Pixel-pair form for tiny channel counts under stride 2 (a network's first layer): pad the
+        // channels to 4 and read two horizontally adjacent pixels as one 8-channel pixel.  The
+        // convolution then has ceil((kw + shift) / 2) horizontal taps, horizontal stride 1 and left
+        // padding (pad + shift) / 2 with shift = pad & 1, each filter row of a window is one
+        // contiguous run of memory, and K shrinks (7x7x3: 224 instead of 392 with 8-channel padding).
+        const bool pairs = (L->C_in <= 4 && L->stride == 2 && (W % 2) == 0);
+        const int Cp = pairs ? 4 : (L->C_in + 7) / 8 * 8;
+        const int shift = pairs ? (L->pad & 1) : 0;
+        const int kw2 = pairs ? (L->kw + shift + 1) / 2 : L->kw;
+        const int Ck = pairs ? 8 : Cp;                                     // channels the kernel sees
+        const int64_t pixels = (int64_t)Nb * H * W, taps = (int64_t)L->C_out * L->kh * kw2;
         if (pixels * Cp > lim) return ASX_ERR_UNSUPPORTED;
-        const size_t need_x = (size_t)pixels * Cp * 2, need_w = (size_t)taps * Cp * 2;
+        const size_t need_x = (size_t)pixels * Cp * 2, need_w = (size_t)taps * Ck * 2;
         if (need_x > L->xpad_bytes || need_w > L->wpack_bytes) {
             cudaStreamSynchronize(st);
             if (need_x > L->xpad_bytes) {
@@ -311,12 +321,20 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
             L->tmap_ptr = nullptr;
         }
         cudaError_t e = launch_pad_channels(x, L->d_xpad, pixels, L->C_in, Cp, st);
-        if (e == cudaSuccess) e = launch_pad_channels(w, L->d_wpack, taps, L->C_in, Cp, st);
+        if (e == cudaSuccess)
+            e = pairs ? launch_pack_pair_filters(w, L->d_wpack, L->C_out, L->kh, L->kw, L->C_in, kw2, shift, st)
+                      : launch_pad_channels(w, L->d_wpack, (int64_t)L->C_out * L->kh * L->kw, L->C_in, Cp, st);
         if (e != cudaSuccess) return from_cuda(e);
         xsrc = L->d_xpad;
         wsrc = L->d_wpack;
-        g.C_in = Cp;
-        g.K = L->kh * L->kw * Cp;
+        g.C_in = Ck;
+        g.kw = kw2;
+        g.K = L->kh * kw2 * Ck;
+        if (pairs) {
+            g.W = W / 2;
+            g.stride_w = 1;
+            g.pad_w = (L->pad + shift) / 2;
+        }
     }
     FastPlan plan;
     long long est_rows = M;                                       // unknown on the host: assume every row kept

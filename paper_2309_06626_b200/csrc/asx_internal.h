@@ -10,6 +10,8 @@ namespace asx {
 // Geometry of one call, passed by value to the kernels.
 struct ConvGeom {
     int Nb, H, W, C_in, C_out, kh, kw, stride, pad, Ho, Wo;
+    int stride_w, pad_w;   // horizontal stride and left padding (equal to stride, pad unless the host
+                           // re-expressed the input as pixel pairs)
     int K;            // kh*kw*C_in
     int P;            // Ho*Wo
     int M;            // Nb*P
@@ -67,7 +69,11 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
                         const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
                         int num_sms, cudaStream_t st);
-// src[rows][C] -> dst[rows][Cp] with zero channels added (Cp a multiple of 8)
+// src[rows][C] -> dst[rows][Cp] with zero channels added (Cp = 4 or a multiple of 8; rows*Cp % 8 == 0)
 cudaError_t launch_pad_channels(const void* src, void* dst, long long rows, int C, int Cp, cudaStream_t st);
+// filters for the pixel-pair form: w[C_out][kh][kw][C] -> w2[C_out][kh][kw2][2][4], where pair kxx,
+// half j holds the original tap kx = 2*kxx + j - shift (zero when outside 0..kw-1 or c >= C)
+cudaError_t launch_pack_pair_filters(const void* w, void* w2, int C_out, int kh, int kw, int C, int kw2, int shift,
+                                     cudaStream_t st);
 
 }  // namespace asx

@@ -226,7 +226,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                     if (row < g.M) {
                         const int n = row / g.P, p = row - n * g.P;
                         const int oy = p / g.Wo, ox = p - oy * g.Wo;
-                        const int iy0 = oy * g.stride - g.pad, ix0 = ox * g.stride - g.pad;
+                        const int iy0 = oy * g.stride - g.pad, ix0 = ox * g.stride_w - g.pad_w;
                         info.x = (n * g.H + iy0) * g.W + ix0;
                         info.y = (iy0 << 16) | (ix0 & 0xffff);
                     } else {
@@ -525,29 +525,50 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     }
 }
 
-// Channel padding: src[rows][C] -> dst[rows][Cp], Cp a multiple of 8, zeros in the added channels.
-// Used for inputs and filters whose channel count is not a multiple of 8, so that every filter
-// tap of a pixel is a whole number of 16-byte chunks.  One thread per 16-byte chunk of dst.
+// Channel padding: src[rows][C] -> dst[rows][Cp] with zeros in the added channels, Cp = 4 or a
+// multiple of 8.  Used for inputs and filters whose channel count is not a multiple of 8, so that
+// the gather can work in 16-byte chunks.  One thread per 16-byte chunk (8 elements) of dst.
 __global__ void pad_channels_kernel(const unsigned short* __restrict__ src, uint4* __restrict__ dst,
                                     long long rows, int C, int Cp)
 {
     ptx::grid_launch_dependents();
     ptx::grid_dependency_wait();
-    const int cpr = Cp >> 3;
-    const long long total = rows * cpr;
+    const long long total = rows * Cp / 8;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
-        const long long row = i / cpr;
-        const int c0 = (int)(i - row * cpr) * 8;
+        long long row = (i * 8) / Cp;
+        int c = (int)((i * 8) - row * Cp);
         unsigned short e[8];
 #pragma unroll
-        for (int q2 = 0; q2 < 8; ++q2) e[q2] = (c0 + q2 < C) ? src[row * C + c0 + q2] : (unsigned short)0;
+        for (int q2 = 0; q2 < 8; ++q2) {
+            e[q2] = (c < C) ? src[row * C + c] : (unsigned short)0;
+            if (++c == Cp) { c = 0; ++row; }
+        }
         uint4 v;
         v.x = e[0] | ((uint32_t)e[1] << 16);
         v.y = e[2] | ((uint32_t)e[3] << 16);
         v.z = e[4] | ((uint32_t)e[5] << 16);
         v.w = e[6] | ((uint32_t)e[7] << 16);
         dst[i] = v;
+    }
+}
+
+// Filters of the pixel-pair form (see asx_run): one thread per output element.
+__global__ void pack_pair_filters_kernel(const unsigned short* __restrict__ w, unsigned short* __restrict__ w2,
+                                         int C_out, int kh, int kw, int C, int kw2, int shift)
+{
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
+    const long long total = (long long)C_out * kh * kw2 * 8;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i & 3), j = (int)((i >> 2) & 1);
+        long long rest = i >> 3;
+        const int kxx = (int)(rest % kw2); rest /= kw2;
+        const int ky = (int)(rest % kh);
+        const int co = (int)(rest / kh);
+        const int kx = 2 * kxx + j - shift;
+        w2[i] = (kx >= 0 && kx < kw && c < C) ? w[(((long long)co * kh + ky) * kw + kx) * C + c] : (unsigned short)0;
     }
 }
 
@@ -629,11 +650,21 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
 
 cudaError_t launch_pad_channels(const void* src, void* dst, long long rows, int C, int Cp, cudaStream_t st)
 {
-    const long long total = rows * (Cp / 8);
+    const long long total = rows * Cp / 8;
     int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     if (blocks < 1) blocks = 1;
     return launch_pdl(pad_channels_kernel, dim3(blocks), dim3(256), 0, st, static_cast<const unsigned short*>(src),
                       static_cast<uint4*>(dst), rows, C, Cp);
+}
+
+cudaError_t launch_pack_pair_filters(const void* w, void* w2, int C_out, int kh, int kw, int C, int kw2, int shift,
+                                     cudaStream_t st)
+{
+    const long long total = (long long)C_out * kh * kw2 * 8;
+    int blocks = (int)((total + 255) / 256 < 1024 ? (total + 255) / 256 : 1024);
+    if (blocks < 1) blocks = 1;
+    return launch_pdl(pack_pair_filters_kernel, dim3(blocks), dim3(256), 0, st, static_cast<const unsigned short*>(w),
+                      static_cast<unsigned short*>(w2), C_out, kh, kw, C, kw2, shift);
 }
 
 }  // namespace asx
