@@ -34,7 +34,8 @@ static_assert(BK == 64, "the MMA loop issues four K=16 instructions per stage");
 constexpr int MAX_STAGES = 8;
 constexpr int MIN_STAGES = 4;
 constexpr int WARP_TMA = 0, WARP_MMA = 1, WARP_EPI0 = 2, WARP_PROD0 = 6;
-constexpr int NUM_PROD_WARPS = 8, NUM_EPI_WARPS = 4;
+constexpr int NUM_PROD_WARPS = 16, NUM_EPI_WARPS = 4;
+constexpr int GROUP_WARPS = 8;          // gather warps per group: 8 warps x 16 rows = one 128-row stage
 constexpr int INFO_RING = 8;            // tiles whose row coordinates are kept in shared memory (power of two)
 constexpr int WARP_ZERO0 = WARP_PROD0 + NUM_PROD_WARPS, NUM_ZERO_WARPS = 4;
 constexpr int WARP_INFO = WARP_ZERO0 + NUM_ZERO_WARPS;
@@ -142,7 +143,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         for (int s = 0; s < S; ++s) {
             // the filter thread's expect_tx arrival (which in TMA mode also announces the gathered
             // bytes) + in the copy modes every gather lane's arrival
-            ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1 + (MODE == GATHER_TMA ? 0 : NUM_PROD_WARPS * 32));
+            ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1 + (MODE == GATHER_TMA ? 0 : GROUP_WARPS * 32));
             ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), 1);
         }
         for (int i = 0; i < INFO_RING; ++i) {
@@ -406,54 +407,53 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         }
     } else {
         // ------------------------------------------------------------------ gather producers
-        // Every warp takes part in every stage and owns 16 of the tile's 128 rows.  The rows'
-        // coordinates are read from the shared-memory ring once per tile; the k loop then only
-        // forms addresses and issues copies, whose completion is reported to the stage's mbarrier
-        // asynchronously, so the warps run ahead of the tensor core by up to S stages.
+        // Two groups of eight warps take the pipeline stages in turn (stage it belongs to group
+        // it % 2); within a group each warp owns 16 of the tile's 128 rows.  The rows' coordinates
+        // are read from the shared-memory ring once per tile; the k loop then only forms addresses
+        // and issues copies whose completion is reported to the stage's mbarrier asynchronously, so
+        // the warps run ahead of the tensor core by up to S stages.  With narrow tiles the loop is
+        // bound by how fast one warp gets through an iteration, hence the two groups.
         const int pw = warp - WARP_PROD0;
+        const int grp = pw / GROUP_WARPS, pwg = pw - grp * GROUP_WARPS;
         const unsigned short* x2 = reinterpret_cast<const unsigned short*>(a.x);
-        const int c = lane & 7;                        // 16-byte chunk of the 128-byte row (copy modes)
-        const int rq = lane >> 3;                      // copy modes: rows 16pw + rq + {0,4,8,12}
-        const int oob = g.Nb * g.H * g.W;              // TMA mode: a row index past the tensor reads zeros
         if (MODE == GATHER_TMA) {
-            // Lanes 0..3 of each warp run the whole loop on their own: each fetches four rows per
-            // stage with one TMA row gather (one 64-channel slice of one filter tap per stage;
-            // padding taps point past the end of the tensor and read zeros).  The bytes are
-            // announced to the stage's barrier by the filter thread, so nothing here needs the
-            // other lanes, and the next stage's row indices are formed before waiting for its slot.
+            // Lanes 0..3 of each warp run the loop on their own: each fetches four rows per stage
+            // with one TMA row gather (one 64-channel slice of one filter tap per stage; padding
+            // taps point past the end of the tensor and read zeros).  The bytes are announced to
+            // the stage's barrier by the filter thread.  A row gather costs its warp about 100
+            // cycles plus 56 per further lane, hence few issuing lanes in many warps.
             if (lane < 4) {
-                int s = 0, j = 0;
+                const int oob = g.Nb * g.H * g.W;
+                int s = 0, j = 0, it = 0;
                 uint32_t ph = 0;
                 bool ok = true;
                 for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++j) {
                     const int r = j & (INFO_RING - 1);
                     if (!wait_bar<100>(ptx::smem_u32(&sh->info_full[r]), (uint32_t)(j / INFO_RING) & 1u, abort_flag, a.dev_status)) break;
-                    const int2* info = sh->rowinfo[r] + 16 * pw + 4 * lane;
+                    const int2* info = sh->rowinfo[r] + 16 * pwg + 4 * lane;
                     const int4 ra = *reinterpret_cast<const int4*>(info);
                     const int4 rb = *reinterpret_cast<const int4*>(info + 2);
                     const int pix[4] = {ra.x, ra.z, rb.x, rb.z}, yx[4] = {ra.y, ra.w, rb.y, rb.w};
                     __syncwarp(0xfu);
                     if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));    // the ring slot is in registers now
                     int ky = 0, kx = 0, ci = 0;
-                    auto indices = [&](int (&idx)[4]) {
-                        const int koff = ky * g.W + kx;
+                    for (int kb = 0; kb < KB; ++kb, ++it) {
+                        if ((it & 1) == grp) {
+                            const int koff = ky * g.W + kx;
+                            int idx[4];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
-                            idx[i] = ((unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W) ? pix[i] + koff : oob;
+                            for (int i = 0; i < 4; ++i) {
+                                const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
+                                idx[i] = ((unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W) ? pix[i] + koff : oob;
+                            }
+                            if (!wait_bar<20>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
+                            ptx::tma_gather4_2d(smem_base + s * stage_bytes + (uint32_t)(16 * pwg + 4 * lane) * 128u, &tmap_x,
+                                                ptx::smem_u32(&sh->full[s]), ci, idx[0], idx[1], idx[2], idx[3]);
                         }
-                    };
-                    int idx[4];
-                    indices(idx);
-                    for (int kb = 0; kb < KB; ++kb) {
-                        if (!wait_bar<20>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
-                        ptx::tma_gather4_2d(smem_base + s * stage_bytes + (uint32_t)(16 * pw + 4 * lane) * 128u, &tmap_x,
-                                            ptx::smem_u32(&sh->full[s]), ci, idx[0], idx[1], idx[2], idx[3]);
                         ci += BK;                          // next 64 channels, or the next tap
                         if (ci >= g.C_in) {
                             ci = 0;
                             if (++kx == g.kw) { kx = 0; ++ky; }
-                            indices(idx);
                         }
                         if (++s == S) { s = 0; ph ^= 1u; }
                     }
@@ -461,59 +461,60 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             }
             __syncwarp();
         } else {
-        int s = 0, j = 0;
-        uint32_t ph = 0;
-        bool ok = true;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++j) {
-            const int r = j & (INFO_RING - 1);
-            if (!warp_wait_bar<100>(ptx::smem_u32(&sh->info_full[r]), (uint32_t)(j / INFO_RING) & 1u, abort_flag, a.dev_status)) break;
-            const int2* info = sh->rowinfo[r] + 16 * pw;
-            int pix[4], yx[4];
+            const int c = lane & 7;                        // 16-byte chunk of the 128-byte row
+            const int rq = lane >> 3;                      // rows 16pwg + rq + {0,4,8,12}
+            int s = 0, j = 0, it = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++j) {
+                const int r = j & (INFO_RING - 1);
+                if (!warp_wait_bar<100>(ptx::smem_u32(&sh->info_full[r]), (uint32_t)(j / INFO_RING) & 1u, abort_flag, a.dev_status)) break;
+                const int2* info = sh->rowinfo[r] + 16 * pwg;
+                int pix[4], yx[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int2 ri = info[rq + 4 * i];
-                pix[i] = ri.x; yx[i] = ri.y;
-            }
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));    // the ring slot is in registers now
+                for (int i = 0; i < 4; ++i) {
+                    const int2 ri = info[rq + 4 * i];
+                    pix[i] = ri.x; yx[i] = ri.y;
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));    // the ring slot is in registers now
 
-            // window position of this lane's first K element of the stage
-            int ky, kx, ci;
-            {
-                const int k_first = c * 8;
-                const int tap = k_first / g.C_in;
-                ci = k_first - tap * g.C_in;
-                ky = tap / g.kw;
-                kx = tap - ky * g.kw;
-            }
-            for (int kb = 0; kb < KB; ++kb) {
-                if (!warp_wait_bar<40>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
-                const uint32_t full = ptx::smem_u32(&sh->full[s]);
-                const uint32_t stage = smem_base + s * stage_bytes + (uint32_t)(16 * pw) * 128u;
+                // window position (filter tap and channel) of this lane's first K element of the stage
+                int ky, kx, ci;
                 {
-                    const bool kvalid = ky < g.kh;     // past K: the window is exhausted
-                    const int koff = ky * g.W + kx;
+                    const int k_first = c * 8;
+                    const int tap = k_first / g.C_in;
+                    ci = k_first - tap * g.C_in;
+                    ky = tap / g.kw;
+                    kx = tap - ky * g.kw;
+                }
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    if ((it & 1) == grp) {
+                        if (!warp_wait_bar<40>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
+                        const uint32_t stage = smem_base + s * stage_bytes + (uint32_t)(16 * pwg) * 128u;
+                        const bool kvalid = ky < g.kh;     // past K: the window is exhausted
+                        const int koff = ky * g.W + kx;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int row = rq + 4 * i;    // row & 7 == (rq + 4i) & 7
-                        const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
-                        const bool in = kvalid && (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
-                        const unsigned short* src = in ? x2 + ((long long)(pix[i] + koff) * g.C_in + ci) : x2;
-                        ptx::cp_async_16(stage + (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)), src, in ? 16u : 0u);
+                        for (int i = 0; i < 4; ++i) {
+                            const int row = rq + 4 * i;    // (16pwg + row) & 7 == row & 7
+                            const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
+                            const bool in = kvalid && (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
+                            const unsigned short* src = in ? x2 + ((long long)(pix[i] + koff) * g.C_in + ci) : x2;
+                            ptx::cp_async_16(stage + (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)), src, in ? 16u : 0u);
+                        }
+                        ptx::cp_async_mbar_arrive_noinc(ptx::smem_u32(&sh->full[s]));
                     }
-                    ptx::cp_async_mbar_arrive_noinc(full);
+                    // advance the window position by 64 K elements
+                    ci += BK;
+                    while (ci >= g.C_in) {
+                        ci -= g.C_in;
+                        if (++kx == g.kw) { kx = 0; ++ky; }
+                    }
+                    if (++s == S) { s = 0; ph ^= 1u; }
                 }
-                // advance the window position by 64 K elements
-                ci += BK;
-                while (ci >= g.C_in) {
-                    ci -= g.C_in;
-                    if (++kx == g.kw) { kx = 0; ++ky; }
-                }
-                if (++s == S) { s = 0; ph ^= 1u; }
             }
+            ptx::cp_async_wait<0>();              // nothing of this thread is in flight at exit
         }
-        }
-        if (MODE == GATHER_CPASYNC) ptx::cp_async_wait<0>();      // nothing of this thread is in flight at exit
     }
 
     ptx::tc_fence_before_sync();
@@ -579,9 +580,12 @@ bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, FastPlan
     const int N = g.C_out;
     const int KB = (g.K + BK - 1) / BK;
     const long long m_tiles = (est_kept_rows + BM - 1) / BM > 0 ? (est_kept_rows + BM - 1) / BM : 1;
-    // Tile width: the widest tile (up to 256 columns) does the most work per gathered byte, but
-    // a layer with few kept rows then has fewer tiles than SMs.  Pick the width with the lowest
-    // estimated time = waves x k-blocks x max(copy issue time, MMA time) per k-block.
+    // Tile width.  The main loop is bound by shared-memory bandwidth (128 bytes per clock): per
+    // 64-wide k-block the gathered A tile (16 KB) and the filter slab (BN x 128 bytes) are written
+    // once and read once by the tensor core, so a k-block costs about 256 + 2*BN clocks (BN = 64:
+    // 0.20 us, 128: 0.27 us, 256: 0.40 us at 1.9 GHz; measured 0.29 us at 128).  A wider tile does
+    // more work per byte, a narrower one gives more tiles when a layer has few kept rows.  Pick
+    // the width with the lowest estimated time = waves x (k-blocks x time per k-block + fixed).
     int best_BN = 0;
     double best_cost = 0.0;
     for (int n_tiles = (N + 255) / 256; ; n_tiles *= 2) {
@@ -589,9 +593,9 @@ bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, FastPlan
         const int BN = ((per + 15) / 16) * 16;
         const int nt = (N + BN - 1) / BN;
         const long long waves = (m_tiles * nt + num_sms - 1) / num_sms;
-        const double t_kb = 0.2 > BN * 0.0015 ? 0.2 : BN * 0.0015;          // microseconds, rough
-        const double cost = (double)waves * (KB * t_kb + 1.0);
-        if (best_BN == 0 || cost < best_cost * 0.98) { best_BN = BN; best_cost = cost; }
+        const double t_kb = (256.0 + 2.0 * BN) / 1900.0;                    // microseconds
+        const double cost = (double)waves * (KB * t_kb + 2.0);
+        if (best_BN == 0 || cost < best_cost * 0.97) { best_BN = BN; best_cost = cost; }
         if (BN <= 64) break;
     }
     const int BN = best_BN;
