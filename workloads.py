@@ -255,6 +255,13 @@ def iter_small_cases() -> Iterator[LayerSpec]:
         ("t_3x3_c256", 256, 256, 3, 1, 1, 14, 14, 2, 50, 4),
         ("t_3x3_c5_n7", 5, 7, 3, 1, 1, 12, 11, 2, 30, 1),
         ("t_3x3_c512", 512, 512, 3, 1, 1, 7, 7, 4, 50, 4),
+        # tiny channel counts under stride 2: even width (pixel pairs, odd and even padding),
+        # odd width (plain channel padding), and stride 1
+        ("t_3x3_c3_s2_oddw", 3, 16, 3, 2, 1, 33, 41, 2, 40, 2),
+        ("t_5x5_c4_s2_p2", 4, 24, 5, 2, 2, 30, 32, 2, 30, 1),
+        ("t_2x2_c1_s2_p0", 1, 8, 2, 2, 0, 16, 16, 3, 50, 1),
+        ("t_4x4_c2_s2_p1", 2, 40, 4, 2, 1, 18, 22, 2, 25, 4),
+        ("t_3x3_c4_s1", 4, 16, 3, 1, 1, 14, 15, 2, 50, 1),
     ]
     for i, (name, cin, cout, k, s, p, H, W, Nb, pct, blk) in enumerate(cases):
         yield LayerSpec(name, cin, cout, k, k, s, p, H, W, Nb, pct, blk, "relu",
