@@ -274,7 +274,11 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     L->last_stream = st;
-    if (flags & ASX_RECOMPACT) {
+    // Small masks are compacted inside the fused kernel itself (one launch instead of two); the
+    // reference kernel and large masks take the stand-alone compaction kernel.
+    const bool fuse_compact = (flags & ASX_RECOMPACT) && !(flags & ASX_IMPL_NAIVE) &&
+                              L->rows <= COMPACT_SMALL_MAX_ROWS;
+    if ((flags & ASX_RECOMPACT) && !fuse_compact) {
         s = run_compaction(L, st);
         if (s != ASX_OK) return s;
     }
@@ -339,7 +343,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     FastPlan plan;
     long long est_rows = M;                                       // unknown on the host: assume every row kept
     if (L->host_kept >= 0) est_rows = (L->rows == P) ? L->host_kept * Nb : L->host_kept;
-    if (!plan_fast(g, L->num_sms, est_rows, &plan)) return ASX_ERR_UNSUPPORTED;
+    if (!plan_fast(g, L->num_sms, est_rows, fuse_compact ? (int)L->rows : 0, &plan)) return ASX_ERR_UNSUPPORTED;
     const int Kw = g.K;
     if (L->tmap_ptr != wsrc || L->tmap_BN != plan.BN || L->tmap_Kw != Kw) {
         EncodeTiledFn enc = encode_tiled_fn();
@@ -371,7 +375,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         }
     }
     return from_cuda(launch_fast(g, plan, L->tmap, plan.vec == 2 ? L->tmap_x : L->tmap, xsrc, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
-                                 L->num_sms, st));
+                                 L->num_sms, fuse_compact ? 1 : 0, st));
 }
 
 asx_status asx_get_kept(asx_layer* L, int64_t* count, const int32_t** dev_kept)

@@ -53,6 +53,9 @@ struct FastArgs {
     int relu;
     int BN, n_tiles, stages, tmem_cols;
     int vec_out;        // C_out % 8 == 0 and y 16-byte aligned: 16-byte stores
+    int fuse_compact;   // rebuild the kept-row list from the mask inside this kernel (small masks)
+    int32_t* kept_out;  // where the fused compaction writes the list and its count
+    int32_t* count_out;
 };
 
 struct alignas(16) Shared {           // lives after the operand stages
@@ -66,6 +69,7 @@ struct alignas(16) Shared {           // lives after the operand stages
     unsigned long long acc_empty[2];
     unsigned int tmem_base;
     int abort;
+    int scan_total[32];   // fused compaction: kept rows per warp
 };
 
 // Bounded wait on an mbarrier phase.  The waiter is suspended by the hardware between polls
@@ -100,14 +104,73 @@ __device__ __forceinline__ bool warp_wait_bar(uint32_t bar, uint32_t parity, vol
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
+// S1 inside the fused kernel, for masks of at most 16384 rows: the whole block scans the mask
+// (16 bytes per thread, popcount, shuffle scan within the warps, warp totals through shared
+// memory) and writes the ascending kept positions as 16-bit values into its own shared memory;
+// block 0 also writes the list to global memory (every block writing the same global addresses
+// serialises in L2 and cost 10-20 us).  Returns the count.
+__device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, int rows, unsigned short* kept_s,
+                                             int32_t* kept_g, int* scan_total, int nthreads)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = nthreads >> 5;
+    int running = 0;
+    for (int base = 0; base < rows; base += nthreads * 16) {
+        const int first = base + tid * 16;
+        unsigned flags = 0;
+        if (first + 16 <= rows && (reinterpret_cast<uintptr_t>(mask) & 15) == 0) {
+            const uint4 v = *reinterpret_cast<const uint4*>(mask + first);
+            const unsigned w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int q2 = 0; q2 < 4; ++q2) {
+                const unsigned t = ((w4[q2] & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w4[q2];      // bit 7 of each byte: byte != 0
+                flags |= (((t >> 7) & 1u) | ((t >> 14) & 2u) | ((t >> 21) & 4u) | ((t >> 28) & 8u)) << (4 * q2);
+            }
+        } else {
+            for (int q2 = 0; q2 < 16; ++q2)
+                if (first + q2 < rows && mask[first + q2] != 0) flags |= 1u << q2;
+        }
+        const int mine = __popc(flags);
+        int incl = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += t;
+        }
+        if (lane == 31) scan_total[warp] = incl;
+        __syncthreads();
+        int prefix = 0, total = 0;
+        for (int i = 0; i < nwarps; ++i) {
+            const int t = scan_total[i];
+            if (i < warp) prefix += t;
+            total += t;
+        }
+        int at = running + prefix + incl - mine;
+        while (flags) {
+            const int q2 = __ffs(flags) - 1;
+            flags &= flags - 1;
+            kept_s[at] = (unsigned short)(first + q2);
+            if (kept_g != nullptr) kept_g[at] = first + q2;
+            ++at;
+        }
+        running += total;
+        __syncthreads();
+    }
+    return running;
+}
+
 // Output row (n*P + p) of the rk-th kept lowered row.
-__device__ __forceinline__ int out_row_of(int rk, int cnt, const ConvGeom& g, const int32_t* __restrict__ kept)
+struct KeptList {
+    const int32_t* g;            // in global memory, or
+    const unsigned short* s;     // this block's 16-bit copy in shared memory (fused compaction)
+    __device__ __forceinline__ int at(int i) const { return s != nullptr ? (int)s[i] : __ldg(g + i); }
+};
+__device__ __forceinline__ int out_row_of(int rk, int cnt, const ConvGeom& g, const KeptList& kept)
 {
     if (g.rows == g.P) {
         const int n = rk / cnt;
-        return n * g.P + __ldg(kept + (rk - n * cnt));
+        return n * g.P + kept.at(rk - n * cnt);
     }
-    return __ldg(kept + rk);
+    return kept.at(rk);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
@@ -173,7 +236,16 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     // From here on the kernel reads what earlier kernels wrote (the kept-row list and its count,
     // the input) and writes the output, so it waits for them to have finished.
     ptx::grid_dependency_wait();
-    const int cnt = *a.count;
+    int cnt;
+    KeptList kept_list{a.kept, nullptr};
+    if (a.fuse_compact) {
+        unsigned short* kept_s = reinterpret_cast<unsigned short*>(sh + 1);     // after the barriers
+        cnt = block_compact(a.mask, g.rows, kept_s, blockIdx.x == 0 ? a.kept_out : nullptr, sh->scan_total, NUM_THREADS);
+        if (blockIdx.x == 0 && tid == 0) *a.count_out = cnt;
+        kept_list.s = kept_s;
+    } else {
+        cnt = *a.count;
+    }
     const int Mk = (g.rows == g.P) ? g.Nb * cnt : cnt;
     // With every position dropped there are no tiles; the zero warps then write the whole output
     // (Algorithm 2, mask == 0 branch).
@@ -217,7 +289,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
 #pragma unroll
             for (int q2 = 0; q2 < 4; ++q2) {
                 const int rk = m_tile * BM + lane * 4 + q2;
-                orow[q2] = (rk < Mk) ? out_row_of(rk, cnt, g, a.kept) : -1;
+                orow[q2] = (rk < Mk) ? out_row_of(rk, cnt, g, kept_list) : -1;
             }
 #pragma unroll
             for (int q2 = 0; q2 < 4; ++q2) {
@@ -293,7 +365,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             const uint32_t use = (uint32_t)(ti >> 1) & 1u;
             const int rk = m_tile * BM + q * 32 + lane;
             const bool valid = rk < Mk;
-            const long long yoff = valid ? (long long)out_row_of(rk, cnt, g, a.kept) * N : 0;
+            const long long yoff = valid ? (long long)out_row_of(rk, cnt, g, kept_list) * N : 0;
             {
                 float* sb = sh->bias[buf];
                 const int et = (warp - WARP_EPI0) * 32 + lane;
@@ -575,7 +647,7 @@ __global__ void pack_pair_filters_kernel(const unsigned short* __restrict__ w, u
 
 }  // namespace
 
-bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, FastPlan* plan)
+bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fused_list_rows, FastPlan* plan)
 {
     const int N = g.C_out;
     const int KB = (g.K + BK - 1) / BK;
@@ -601,14 +673,15 @@ bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, FastPlan
     const int BN = best_BN;
     const int n_tiles = (N + BN - 1) / BN;
     const int stage_bytes = A_STAGE_BYTES + BN * BK * 2;
-    const int budget = 227 * 1024 - 1024 - (int)sizeof(Shared);
+    const int list_bytes = (fused_list_rows * 2 + 15) / 16 * 16;     // 16-bit kept list of the fused compaction
+    const int budget = 227 * 1024 - 1024 - (int)sizeof(Shared) - list_bytes;
     int S = budget / stage_bytes;
     if (S > MAX_STAGES) S = MAX_STAGES;
     if (S < MIN_STAGES) return false;
     plan->BN = BN;
     plan->n_tiles = n_tiles;
     plan->stages = S;
-    int smem = 1024 + S * stage_bytes + (int)sizeof(Shared);
+    int smem = 1024 + S * stage_bytes + (int)sizeof(Shared) + list_bytes;
     if (smem < 120 * 1024) smem = 120 * 1024;      // one block per SM: tensor memory is not shared out
     plan->smem_bytes = smem;
     if (g.C_in % 8 != 0) return false;            // the caller pads the channels first
@@ -620,9 +693,12 @@ bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, FastPlan
 cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorMap& tmap_w,
                         const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
-                        int num_sms, cudaStream_t st)
+                        int num_sms, int fuse_compact, cudaStream_t st)
 {
     FastArgs a;
+    a.fuse_compact = fuse_compact;
+    a.kept_out = const_cast<int32_t*>(kept);
+    a.count_out = const_cast<int32_t*>(count);
     a.x = static_cast<const __nv_bfloat16*>(x);
     a.bias = bias;
     a.y = static_cast<__nv_bfloat16*>(y);

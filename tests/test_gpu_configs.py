@@ -27,8 +27,7 @@ def _check_layer(spec, rng):
     y.view(torch.int16).fill_(0x7fc1)                                   # NaN canary: every element must be written
     layer = asx.MaskedConvLayer(spec.C_in, spec.C_out, spec.kh, spec.kw, spec.stride, spec.pad)
     layer.set_mask(mask)
-    layer.recompact()
-    layer.run(xd, wd, bd, out=y, flags=asx.ACT_RELU)
+    layer.run(xd, wd, bd, out=y, flags=asx.ACT_RELU | asx.RECOMPACT)
     torch.cuda.synchronize()
     assert layer.device_status() == 0
     kept = layer.kept()
