@@ -42,7 +42,34 @@ constexpr int WARP_INFO = WARP_ZERO0 + NUM_ZERO_WARPS;
 constexpr int NUM_THREADS = 32 * (WARP_INFO + 1);
 constexpr long long WAIT_CYCLE_LIMIT = 4000000000ll;   // about two seconds
 
+// Division of a 32-bit unsigned number by a divisor fixed for the whole launch, as a multiply-high
+// and two shifts (Granlund and Montgomery's round-up method: l = ceil(log2 d),
+// m = floor(2^32 (2^l - d) / d) + 1, q = (t + ((n - t) >> min(l,1))) >> max(l-1,0) with
+// t = mulhi(m, n); exact for every n < 2^32 and 1 <= d < 2^31).  A hardware-less 32-bit division
+// is about 35 dependent instructions, and the row-coordinate warp did twelve per tile.
+struct FastDiv {
+    uint32_t d, m, s1, s2;
+};
+__host__ __device__ inline FastDiv make_fastdiv(uint32_t d)
+{
+    uint32_t l = 0;
+    while ((1ull << l) < d) ++l;
+    const unsigned long long m = ((((1ull << l) - d) << 32) / d) + 1ull;
+    FastDiv f;
+    f.d = d;
+    f.m = (uint32_t)m;
+    f.s1 = l ? 1u : 0u;
+    f.s2 = l ? l - 1u : 0u;
+    return f;
+}
+__device__ __forceinline__ uint32_t fd_div(uint32_t n, const FastDiv& f)
+{
+    const uint32_t t = __umulhi(f.m, n);
+    return (t + ((n - t) >> f.s1)) >> f.s2;
+}
+
 struct FastArgs {
+    FastDiv fdP, fdWo;           // divisions by P and Wo
     const __nv_bfloat16* x;
     const float* bias;
     __nv_bfloat16* y;
@@ -106,11 +133,11 @@ __device__ __forceinline__ bool warp_wait_bar(uint32_t bar, uint32_t parity, vol
 
 // S1 inside the fused kernel, for masks of at most 16384 rows: the whole block scans the mask
 // (16 bytes per thread, popcount, shuffle scan within the warps, warp totals through shared
-// memory) and writes the ascending kept positions as 16-bit values into its own shared memory;
-// block 0 also writes the list to global memory (every block writing the same global addresses
-// serialises in L2 and cost 10-20 us).  Returns the count.
+// memory) and writes the ascending kept positions as 16-bit values into its own shared memory
+// (every block writing the list to the same global addresses serialises in L2 and cost 10-20 us;
+// block 0 alone copies it out).  Returns the count.
 __device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, int rows, unsigned short* kept_s,
-                                             int32_t* kept_g, int* scan_total, int nthreads)
+                                             int* scan_total, int nthreads)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = nthreads >> 5;
     int running = 0;
@@ -148,9 +175,7 @@ __device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, i
         while (flags) {
             const int q2 = __ffs(flags) - 1;
             flags &= flags - 1;
-            kept_s[at] = (unsigned short)(first + q2);
-            if (kept_g != nullptr) kept_g[at] = first + q2;
-            ++at;
+            kept_s[at++] = (unsigned short)(first + q2);
         }
         running += total;
         __syncthreads();
@@ -164,11 +189,11 @@ struct KeptList {
     const unsigned short* s;     // this block's 16-bit copy in shared memory (fused compaction)
     __device__ __forceinline__ int at(int i) const { return s != nullptr ? (int)s[i] : __ldg(g + i); }
 };
-__device__ __forceinline__ int out_row_of(int rk, int cnt, const ConvGeom& g, const KeptList& kept)
+__device__ __forceinline__ int out_row_of(int rk, const FastDiv& fdcnt, const ConvGeom& g, const KeptList& kept)
 {
     if (g.rows == g.P) {
-        const int n = rk / cnt;
-        return n * g.P + kept.at(rk - n * cnt);
+        const int n = (int)fd_div((uint32_t)rk, fdcnt);
+        return n * g.P + kept.at(rk - n * (int)fdcnt.d);
     }
     return kept.at(rk);
 }
@@ -233,16 +258,23 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
 
-    // From here on the kernel reads what earlier kernels wrote (the kept-row list and its count,
-    // the input) and writes the output, so it waits for them to have finished.
-    ptx::grid_dependency_wait();
-    int cnt;
+    // The layer's mask is only ever written by stream-ordered copies, never by a kernel, so the
+    // fused compaction may read it while the preceding kernel is still running.
+    int cnt = 0;
     KeptList kept_list{a.kept, nullptr};
+    unsigned short* kept_s = reinterpret_cast<unsigned short*>(sh + 1);     // after the barriers
     if (a.fuse_compact) {
-        unsigned short* kept_s = reinterpret_cast<unsigned short*>(sh + 1);     // after the barriers
-        cnt = block_compact(a.mask, g.rows, kept_s, blockIdx.x == 0 ? a.kept_out : nullptr, sh->scan_total, NUM_THREADS);
-        if (blockIdx.x == 0 && tid == 0) *a.count_out = cnt;
+        cnt = block_compact(a.mask, g.rows, kept_s, sh->scan_total, NUM_THREADS);
         kept_list.s = kept_s;
+    }
+    // From here on the kernel reads what earlier kernels wrote (the kept-row list and its count,
+    // the input) and writes the output and the list, so it waits for them to have finished.
+    ptx::grid_dependency_wait();
+    if (a.fuse_compact) {
+        if (blockIdx.x == 0) {      // the list in global memory, for asx_get_kept and later runs
+            for (int i = tid; i < cnt; i += NUM_THREADS) a.kept_out[i] = (int32_t)kept_s[i];
+            if (tid == 0) *a.count_out = cnt;
+        }
     } else {
         cnt = *a.count;
     }
@@ -276,6 +308,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         // ------------------------------------------------------------------ row coordinates
         // Decodes the kept rows of upcoming tiles into the shared-memory ring, four rows per lane,
         // running ahead of the gather warps by up to INFO_RING tiles.
+        const FastDiv fdcnt = make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));
         int j = 0;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++j) {
             const int r = j % INFO_RING;
@@ -289,7 +322,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
 #pragma unroll
             for (int q2 = 0; q2 < 4; ++q2) {
                 const int rk = m_tile * BM + lane * 4 + q2;
-                orow[q2] = (rk < Mk) ? out_row_of(rk, cnt, g, kept_list) : -1;
+                orow[q2] = (rk < Mk) ? out_row_of(rk, fdcnt, g, kept_list) : -1;
             }
 #pragma unroll
             for (int q2 = 0; q2 < 4; ++q2) {
@@ -297,8 +330,8 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                 const int row = orow[q2];
                 if (row >= 0) {
                     if (row < g.M) {
-                        const int n = row / g.P, p = row - n * g.P;
-                        const int oy = p / g.Wo, ox = p - oy * g.Wo;
+                        const int n = (int)fd_div((uint32_t)row, a.fdP), p = row - n * g.P;
+                        const int oy = (int)fd_div((uint32_t)p, a.fdWo), ox = p - oy * g.Wo;
                         const int iy0 = oy * g.stride - g.pad, ix0 = ox * g.stride_w - g.pad_w;
                         info.x = (n * g.H + iy0) * g.W + ix0;
                         info.y = (iy0 << 16) | (ix0 & 0xffff);
@@ -355,6 +388,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3;                       // TMEM lanes 32q .. 32q+31 belong to this warp
         unsigned short* y2 = reinterpret_cast<unsigned short*>(a.y);
+        const FastDiv fdcnt = make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));
         int ti = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
@@ -365,7 +399,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             const uint32_t use = (uint32_t)(ti >> 1) & 1u;
             const int rk = m_tile * BM + q * 32 + lane;
             const bool valid = rk < Mk;
-            const long long yoff = valid ? (long long)out_row_of(rk, cnt, g, kept_list) * N : 0;
+            const long long yoff = valid ? (long long)out_row_of(rk, fdcnt, g, kept_list) * N : 0;
             {
                 float* sb = sh->bias[buf];
                 const int et = (warp - WARP_EPI0) * 32 + lane;
@@ -708,6 +742,8 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     a.dev_status = dev_status;
     a.relu = relu;
     a.BN = plan.BN;
+    a.fdP = make_fastdiv((uint32_t)g.P);
+    a.fdWo = make_fastdiv((uint32_t)g.Wo);
     a.n_tiles = plan.n_tiles;
     a.stages = plan.stages;
     int cols = 32;
