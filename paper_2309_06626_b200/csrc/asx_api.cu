@@ -375,7 +375,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         }
     }
     return from_cuda(launch_fast(g, plan, L->tmap, plan.vec == 2 ? L->tmap_x : L->tmap, xsrc, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
-                                 L->num_sms, fuse_compact ? 1 : 0, st));
+                                 L->num_sms, fuse_compact ? 1 : 0, L->host_kept, st));
 }
 
 asx_status asx_get_kept(asx_layer* L, int64_t* count, const int32_t** dev_kept)

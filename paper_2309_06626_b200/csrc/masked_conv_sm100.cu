@@ -70,6 +70,7 @@ __device__ __forceinline__ uint32_t fd_div(uint32_t n, const FastDiv& f)
 
 struct FastArgs {
     FastDiv fdP, fdWo;           // divisions by P and Wo
+    FastDiv fdcnt_host;          // division by the kept count when the host knows it (d = 0: it does not)
     const __nv_bfloat16* x;
     const float* bias;
     __nv_bfloat16* y;
@@ -136,26 +137,35 @@ __device__ __forceinline__ bool warp_wait_bar(uint32_t bar, uint32_t parity, vol
 // memory) and writes the ascending kept positions as 16-bit values into its own shared memory
 // (every block writing the list to the same global addresses serialises in L2 and cost 10-20 us;
 // block 0 alone copies it out).  Returns the count.
-__device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, int rows, unsigned short* kept_s,
-                                             int* scan_total, int nthreads)
+// Bit q of the result: mask[first + q] != 0, for the 16 mask bytes starting at `first`.
+__device__ __forceinline__ unsigned mask_flags16(const uint8_t* __restrict__ mask, int rows, int first)
+{
+    unsigned flags = 0;
+    if (first + 16 <= rows && (reinterpret_cast<uintptr_t>(mask) & 15) == 0) {
+        const uint4 v = *reinterpret_cast<const uint4*>(mask + first);
+        const unsigned w4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int q2 = 0; q2 < 4; ++q2) {
+            const unsigned t = ((w4[q2] & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w4[q2];      // bit 7 of each byte: byte != 0
+            flags |= (((t >> 7) & 1u) | ((t >> 14) & 2u) | ((t >> 21) & 4u) | ((t >> 28) & 8u)) << (4 * q2);
+        }
+    } else {
+        for (int q2 = 0; q2 < 16; ++q2)
+            if (first + q2 < rows && mask[first + q2] != 0) flags |= 1u << q2;
+    }
+    return flags;
+}
+
+// `flags0` are the caller's mask_flags16 of the first pass (first = 16 tid), loaded early so that
+// the latency of the mask read is hidden behind the kernel's set-up.
+__device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, int rows, unsigned flags0,
+                                             unsigned short* kept_s, int* scan_total, int nthreads)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = nthreads >> 5;
     int running = 0;
     for (int base = 0; base < rows; base += nthreads * 16) {
         const int first = base + tid * 16;
-        unsigned flags = 0;
-        if (first + 16 <= rows && (reinterpret_cast<uintptr_t>(mask) & 15) == 0) {
-            const uint4 v = *reinterpret_cast<const uint4*>(mask + first);
-            const unsigned w4[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int q2 = 0; q2 < 4; ++q2) {
-                const unsigned t = ((w4[q2] & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w4[q2];      // bit 7 of each byte: byte != 0
-                flags |= (((t >> 7) & 1u) | ((t >> 14) & 2u) | ((t >> 21) & 4u) | ((t >> 28) & 8u)) << (4 * q2);
-            }
-        } else {
-            for (int q2 = 0; q2 < 16; ++q2)
-                if (first + q2 < rows && mask[first + q2] != 0) flags |= 1u << q2;
-        }
+        unsigned flags = base == 0 ? flags0 : mask_flags16(mask, rows, first);
         const int mine = __popc(flags);
         int incl = mine;
 #pragma unroll
@@ -227,6 +237,11 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
 
     const int KB = (g.K + BK - 1) / BK;
 
+    // The layer's mask is only ever written by stream-ordered copies, never by a kernel, so the
+    // fused compaction may read it while the preceding kernel is still running; the read is
+    // issued first so that its latency overlaps the set-up below.
+    const unsigned flags0 = a.fuse_compact ? mask_flags16(a.mask, g.rows, tid * 16) : 0u;
+
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
             // the filter thread's expect_tx arrival (which in TMA mode also announces the gathered
@@ -258,13 +273,11 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
 
-    // The layer's mask is only ever written by stream-ordered copies, never by a kernel, so the
-    // fused compaction may read it while the preceding kernel is still running.
     int cnt = 0;
     KeptList kept_list{a.kept, nullptr};
     unsigned short* kept_s = reinterpret_cast<unsigned short*>(sh + 1);     // after the barriers
     if (a.fuse_compact) {
-        cnt = block_compact(a.mask, g.rows, kept_s, sh->scan_total, NUM_THREADS);
+        cnt = block_compact(a.mask, g.rows, flags0, kept_s, sh->scan_total, NUM_THREADS);
         kept_list.s = kept_s;
     }
     // From here on the kernel reads what earlier kernels wrote (the kept-row list and its count,
@@ -308,7 +321,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         // ------------------------------------------------------------------ row coordinates
         // Decodes the kept rows of upcoming tiles into the shared-memory ring, four rows per lane,
         // running ahead of the gather warps by up to INFO_RING tiles.
-        const FastDiv fdcnt = make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));
+        const FastDiv fdcnt = (cnt > 0 && a.fdcnt_host.d == (uint32_t)cnt) ? a.fdcnt_host : make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));
         int j = 0;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++j) {
             const int r = j % INFO_RING;
@@ -388,7 +401,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3;                       // TMEM lanes 32q .. 32q+31 belong to this warp
         unsigned short* y2 = reinterpret_cast<unsigned short*>(a.y);
-        const FastDiv fdcnt = make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));
+        const FastDiv fdcnt = (cnt > 0 && a.fdcnt_host.d == (uint32_t)cnt) ? a.fdcnt_host : make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));
         int ti = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
@@ -727,9 +740,11 @@ bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fuse
 cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorMap& tmap_w,
                         const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
-                        int num_sms, int fuse_compact, cudaStream_t st)
+                        int num_sms, int fuse_compact, long long host_kept, cudaStream_t st)
 {
     FastArgs a;
+    a.fdcnt_host = make_fastdiv((uint32_t)(host_kept > 0 && host_kept < (1ll << 31) ? host_kept : 1));
+    if (!(host_kept > 0 && host_kept < (1ll << 31))) a.fdcnt_host.d = 0;
     a.fuse_compact = fuse_compact;
     a.kept_out = const_cast<int32_t*>(kept);
     a.count_out = const_cast<int32_t*>(count);
