@@ -137,35 +137,39 @@ __device__ __forceinline__ bool warp_wait_bar(uint32_t bar, uint32_t parity, vol
 // memory) and writes the ascending kept positions as 16-bit values into its own shared memory
 // (every block writing the list to the same global addresses serialises in L2 and cost 10-20 us;
 // block 0 alone copies it out).  Returns the count.
-// Bit q of the result: mask[first + q] != 0, for the 16 mask bytes starting at `first`.
-__device__ __forceinline__ unsigned mask_flags16(const uint8_t* __restrict__ mask, int rows, int first)
+// Bit q of the result: byte q of the 16 mask bytes in v is non-zero.
+__device__ __forceinline__ unsigned nonzero_bytes16(const uint4& v)
 {
+    const unsigned w4[4] = {v.x, v.y, v.z, v.w};
     unsigned flags = 0;
-    if (first + 16 <= rows && (reinterpret_cast<uintptr_t>(mask) & 15) == 0) {
-        const uint4 v = *reinterpret_cast<const uint4*>(mask + first);
-        const unsigned w4[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int q2 = 0; q2 < 4; ++q2) {
-            const unsigned t = ((w4[q2] & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w4[q2];      // bit 7 of each byte: byte != 0
-            flags |= (((t >> 7) & 1u) | ((t >> 14) & 2u) | ((t >> 21) & 4u) | ((t >> 28) & 8u)) << (4 * q2);
-        }
-    } else {
-        for (int q2 = 0; q2 < 16; ++q2)
-            if (first + q2 < rows && mask[first + q2] != 0) flags |= 1u << q2;
+    for (int q2 = 0; q2 < 4; ++q2) {
+        const unsigned t = ((w4[q2] & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w4[q2];      // bit 7 of each byte: byte != 0
+        flags |= (((t >> 7) & 1u) | ((t >> 14) & 2u) | ((t >> 21) & 4u) | ((t >> 28) & 8u)) << (4 * q2);
     }
     return flags;
 }
+// Bit q of the result: mask[first + q] != 0, for the 16 mask bytes starting at `first`.
+__device__ __forceinline__ unsigned mask_flags16(const uint8_t* __restrict__ mask, int rows, int first)
+{
+    if (first + 16 <= rows && (reinterpret_cast<uintptr_t>(mask) & 15) == 0)
+        return nonzero_bytes16(*reinterpret_cast<const uint4*>(mask + first));
+    unsigned flags = 0;
+    for (int q2 = 0; q2 < 16; ++q2)
+        if (first + q2 < rows && mask[first + q2] != 0) flags |= 1u << q2;
+    return flags;
+}
 
-// `flags0` are the caller's mask_flags16 of the first pass (first = 16 tid), loaded early so that
-// the latency of the mask read is hidden behind the kernel's set-up.
-__device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, int rows, unsigned flags0,
+// `early` holds mask bytes 16 tid .. 16 tid + 15 when `early_ok` (the caller read them before the
+// kernel's set-up so that the latency of the read is hidden behind it).
+__device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, int rows, const uint4& early, bool early_ok,
                                              unsigned short* kept_s, int* scan_total, int nthreads)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = nthreads >> 5;
     int running = 0;
     for (int base = 0; base < rows; base += nthreads * 16) {
         const int first = base + tid * 16;
-        unsigned flags = base == 0 ? flags0 : mask_flags16(mask, rows, first);
+        unsigned flags = (base == 0 && early_ok) ? nonzero_bytes16(early) : mask_flags16(mask, rows, first);
         const int mine = __popc(flags);
         int incl = mine;
 #pragma unroll
@@ -175,12 +179,16 @@ __device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, i
         }
         if (lane == 31) scan_total[warp] = incl;
         __syncthreads();
-        int prefix = 0, total = 0;
-        for (int i = 0; i < nwarps; ++i) {
-            const int t = scan_total[i];
-            if (i < warp) prefix += t;
-            total += t;
+        // every warp scans the (at most 32) warp totals with shuffles
+        const int wt = lane < nwarps ? scan_total[lane] : 0;
+        int winc = wt;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, winc, d);
+            if (lane >= d) winc += t;
         }
+        const int prefix = __shfl_sync(0xffffffffu, winc - wt, warp);
+        const int total = __shfl_sync(0xffffffffu, winc, 31);
         int at = running + prefix + incl - mine;
         while (flags) {
             const int q2 = __ffs(flags) - 1;
@@ -216,6 +224,28 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 
 enum : int { GATHER_CPASYNC = 1, GATHER_TMA = 2 };
 
+// What the gather warps need to know about the rk-th kept lowered row: the pixel index of its
+// window's corner, (n H + iy0) W + ix0, and the corner's coordinates packed as iy0 << 16 | ix0.
+// Rows past the end get iy0 = -32768, for which no filter tap is inside the image.
+__device__ __forceinline__ int2 row_info_of(int rk, int Mk, const FastDiv& fdcnt, const ConvGeom& g, const FastArgs& a,
+                                            const KeptList& kept)
+{
+    int2 info = make_int2(0, (int)0x80000000u);
+    if (rk < Mk) {
+        const int row = out_row_of(rk, fdcnt, g, kept);
+        if (row < g.M) {
+            const int n = (int)fd_div((uint32_t)row, a.fdP), p = row - n * g.P;
+            const int oy = (int)fd_div((uint32_t)p, a.fdWo), ox = p - oy * g.Wo;
+            const int iy0 = oy * g.stride - g.pad, ix0 = ox * g.stride_w - g.pad_w;
+            info.x = (n * g.H + iy0) * g.W + ix0;
+            info.y = (iy0 << 16) | (ix0 & 0xffff);
+        } else {
+            atomicOr(a.dev_status, DEV_BAD_INDEX);
+        }
+    }
+    return info;
+}
+
 template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
@@ -240,7 +270,9 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     // The layer's mask is only ever written by stream-ordered copies, never by a kernel, so the
     // fused compaction may read it while the preceding kernel is still running; the read is
     // issued first so that its latency overlaps the set-up below.
-    const unsigned flags0 = a.fuse_compact ? mask_flags16(a.mask, g.rows, tid * 16) : 0u;
+    uint4 early_mask = make_uint4(0, 0, 0, 0);
+    const bool early_ok = a.fuse_compact && tid * 16 + 16 <= g.rows && (reinterpret_cast<uintptr_t>(a.mask) & 15) == 0;
+    if (early_ok) early_mask = *reinterpret_cast<const uint4*>(a.mask + tid * 16);
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
@@ -277,7 +309,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     KeptList kept_list{a.kept, nullptr};
     unsigned short* kept_s = reinterpret_cast<unsigned short*>(sh + 1);     // after the barriers
     if (a.fuse_compact) {
-        cnt = block_compact(a.mask, g.rows, flags0, kept_s, sh->scan_total, NUM_THREADS);
+        cnt = block_compact(a.mask, g.rows, early_mask, early_ok, kept_s, sh->scan_total, NUM_THREADS);
         kept_list.s = kept_s;
     }
     // From here on the kernel reads what earlier kernels wrote (the kept-row list and its count,
@@ -296,6 +328,19 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     // (Algorithm 2, mask == 0 branch).
     const int m_tiles = (Mk + BM - 1) / BM;
     const int total_tiles = m_tiles * a.n_tiles;
+    const FastDiv fdcnt = (cnt > 0 && a.fdcnt_host.d == (uint32_t)cnt) ? a.fdcnt_host : make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));
+
+    // Row coordinates of this block's first INFO_RING tiles, one row per thread: a single warp
+    // working through them is 1.5 us of dependent arithmetic in front of the first gather.
+    {
+        for (int idx = tid; idx < INFO_RING * BM; idx += NUM_THREADS) {
+            const int jj = idx / BM, rr = idx - jj * BM;
+            const long long t = blockIdx.x + (long long)jj * gridDim.x;
+            if (t < total_tiles) sh->rowinfo[jj][rr] = row_info_of((int)(t / a.n_tiles) * BM + rr, Mk, fdcnt, g, a, kept_list);
+        }
+        __syncthreads();
+        if (tid < INFO_RING && blockIdx.x + (long long)tid * gridDim.x < total_tiles) ptx::mbar_arrive(ptx::smem_u32(&sh->info_full[tid]));
+    }
 
     if (warp == WARP_TMA) {
         // ------------------------------------------------------------------ filter slabs by TMA
@@ -321,38 +366,19 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         // ------------------------------------------------------------------ row coordinates
         // Decodes the kept rows of upcoming tiles into the shared-memory ring, four rows per lane,
         // running ahead of the gather warps by up to INFO_RING tiles.
-        const FastDiv fdcnt = (cnt > 0 && a.fdcnt_host.d == (uint32_t)cnt) ? a.fdcnt_host : make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));
-        int j = 0;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++j) {
+        int j = INFO_RING;                        // the first INFO_RING tiles were decoded by the whole block
+        for (long long t = blockIdx.x + (long long)INFO_RING * gridDim.x; t < total_tiles; t += gridDim.x, ++j) {
             const int r = j % INFO_RING;
             int good = 1;
             if (lane == 0)
                 good = wait_bar<200>(ptx::smem_u32(&sh->info_empty[r]), ((uint32_t)(j / INFO_RING) & 1u) ^ 1u, abort_flag, a.dev_status) ? 1 : 0;
             good = __shfl_sync(0xffffffffu, good, 0);
             if (!good) break;
-            const int m_tile = t / a.n_tiles;
-            int orow[4];
+            const int m_tile = (int)(t / a.n_tiles);
 #pragma unroll
             for (int q2 = 0; q2 < 4; ++q2) {
-                const int rk = m_tile * BM + lane * 4 + q2;
-                orow[q2] = (rk < Mk) ? out_row_of(rk, fdcnt, g, kept_list) : -1;
-            }
-#pragma unroll
-            for (int q2 = 0; q2 < 4; ++q2) {
-                int2 info = make_int2(0, (int)0x80000000u);            // iy0 = -32768: no tap is in bounds
-                const int row = orow[q2];
-                if (row >= 0) {
-                    if (row < g.M) {
-                        const int n = (int)fd_div((uint32_t)row, a.fdP), p = row - n * g.P;
-                        const int oy = (int)fd_div((uint32_t)p, a.fdWo), ox = p - oy * g.Wo;
-                        const int iy0 = oy * g.stride - g.pad, ix0 = ox * g.stride_w - g.pad_w;
-                        info.x = (n * g.H + iy0) * g.W + ix0;
-                        info.y = (iy0 << 16) | (ix0 & 0xffff);
-                    } else {
-                        atomicOr(a.dev_status, DEV_BAD_INDEX);
-                    }
-                }
-                sh->rowinfo[r][lane * 4 + q2] = info;
+                const int rr = lane * 4 + q2;
+                sh->rowinfo[r][rr] = row_info_of(m_tile * BM + rr, Mk, fdcnt, g, a, kept_list);
             }
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_full[r]));
@@ -401,7 +427,6 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3;                       // TMEM lanes 32q .. 32q+31 belong to this warp
         unsigned short* y2 = reinterpret_cast<unsigned short*>(a.y);
-        const FastDiv fdcnt = (cnt > 0 && a.fdcnt_host.d == (uint32_t)cnt) ? a.fdcnt_host : make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));
         int ti = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
