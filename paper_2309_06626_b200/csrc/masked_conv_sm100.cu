@@ -70,6 +70,7 @@ __device__ __forceinline__ uint32_t fd_div(uint32_t n, const FastDiv& f)
 
 struct FastArgs {
     FastDiv fdP, fdWo;           // divisions by P and Wo
+    FastDiv fdNt;                // division by n_tiles
     FastDiv fdcnt_host;          // division by the kept count when the host knows it (d = 0: it does not)
     const __nv_bfloat16* x;
     const float* bias;
@@ -272,7 +273,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     // issued first so that its latency overlaps the set-up below.
     uint4 early_mask = make_uint4(0, 0, 0, 0);
     const bool early_ok = a.fuse_compact && tid * 16 + 16 <= g.rows && (reinterpret_cast<uintptr_t>(a.mask) & 15) == 0;
-    if (early_ok) early_mask = *reinterpret_cast<const uint4*>(a.mask + tid * 16);
+    if (early_ok) early_mask = ptx::ld_global_v4_keep_in_l2(a.mask + tid * 16);
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) {
@@ -328,7 +329,8 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     // (Algorithm 2, mask == 0 branch).
     const int m_tiles = (Mk + BM - 1) / BM;
     const int total_tiles = m_tiles * a.n_tiles;
-    const FastDiv fdcnt = (cnt > 0 && a.fdcnt_host.d == (uint32_t)cnt) ? a.fdcnt_host : make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));
+    FastDiv fdcnt = a.fdcnt_host;
+    if (cnt <= 0 || fdcnt.d != (uint32_t)cnt) fdcnt = make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));   // the host did not know the count
 
     // Row coordinates of this block's first INFO_RING tiles, one row per thread: a single warp
     // working through them is 1.5 us of dependent arithmetic in front of the first gather.
@@ -336,7 +338,8 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         for (int idx = tid; idx < INFO_RING * BM; idx += NUM_THREADS) {
             const int jj = idx / BM, rr = idx - jj * BM;
             const long long t = blockIdx.x + (long long)jj * gridDim.x;
-            if (t < total_tiles) sh->rowinfo[jj][rr] = row_info_of((int)(t / a.n_tiles) * BM + rr, Mk, fdcnt, g, a, kept_list);
+            if (t < total_tiles)
+                sh->rowinfo[jj][rr] = row_info_of((int)fd_div((uint32_t)t, a.fdNt) * BM + rr, Mk, fdcnt, g, a, kept_list);
         }
         __syncthreads();
         if (tid < INFO_RING && blockIdx.x + (long long)tid * gridDim.x < total_tiles) ptx::mbar_arrive(ptx::smem_u32(&sh->info_full[tid]));
@@ -349,7 +352,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             uint32_t ph = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const int n_tile = t % a.n_tiles;
+                const int n_tile = t - (int)fd_div((uint32_t)t, a.fdNt) * a.n_tiles;
                 for (int kb = 0; kb < KB; ++kb) {
                     if (!wait_bar<40>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
                     const uint32_t full = ptx::smem_u32(&sh->full[s]);
@@ -374,7 +377,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                 good = wait_bar<200>(ptx::smem_u32(&sh->info_empty[r]), ((uint32_t)(j / INFO_RING) & 1u) ^ 1u, abort_flag, a.dev_status) ? 1 : 0;
             good = __shfl_sync(0xffffffffu, good, 0);
             if (!good) break;
-            const int m_tile = (int)(t / a.n_tiles);
+            const int m_tile = (int)fd_div((uint32_t)t, a.fdNt);
 #pragma unroll
             for (int q2 = 0; q2 < 4; ++q2) {
                 const int rr = lane * 4 + q2;
@@ -430,7 +433,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         int ti = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
-            const int m_tile = t / a.n_tiles, n_tile = t - m_tile * a.n_tiles;
+            const int m_tile = (int)fd_div((uint32_t)t, a.fdNt), n_tile = t - m_tile * a.n_tiles;
             const int n0 = n_tile * BN;
             // kept rows from the accumulator
             const int buf = ti & 1;
@@ -785,6 +788,7 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     a.fdP = make_fastdiv((uint32_t)g.P);
     a.fdWo = make_fastdiv((uint32_t)g.Wo);
     a.n_tiles = plan.n_tiles;
+    a.fdNt = make_fastdiv((uint32_t)plan.n_tiles);
     a.stages = plan.stages;
     int cols = 32;
     while (cols < 2 * plan.BN) cols <<= 1;

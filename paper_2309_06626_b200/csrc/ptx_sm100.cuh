@@ -121,6 +121,19 @@ __device__ __forceinline__ void st_shared_v4(uint32_t dst, uint4 v)
                  : "memory");
 }
 
+// 16-byte global load that asks L2 to keep the line when it has to evict (for small read-only
+// data that every launch reads first, while the launches in between stream through L2).
+__device__ __forceinline__ uint4 ld_global_v4_keep_in_l2(const void* p)
+{
+    uint64_t pol;
+    uint4 v;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    asm volatile("ld.global.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p), "l"(pol));
+    return v;
+}
+
 // ---------------------------------------------------------------- TMA (tile mode, one CTA)
 __device__ __forceinline__ void prefetch_tensormap(const void* tmap)
 {
