@@ -26,6 +26,10 @@ struct asx_layer {
     // staging copies with zero-padded channels, for C_in not a multiple of 8
     void* d_wpack = nullptr;
     size_t wpack_bytes = 0;
+    void* d_ws = nullptr;              // split-K workspace: fp32 partial tiles, then the tile counters
+    size_t ws_bytes = 0;
+    int* d_wscnt = nullptr;
+    size_t wscnt_ints = 0;
     void* d_xpad = nullptr;
     size_t xpad_bytes = 0;
     // tensor map cache
@@ -343,7 +347,27 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     FastPlan plan;
     long long est_rows = M;                                       // unknown on the host: assume every row kept
     if (L->host_kept >= 0) est_rows = (L->rows == P) ? L->host_kept * Nb : L->host_kept;
-    if (!plan_fast(g, L->num_sms, est_rows, fuse_compact ? (int)L->rows : 0, &plan)) return ASX_ERR_UNSUPPORTED;
+    // Sharing a tile's k-blocks between blocks needs the exact tile count (to size the workspace)
+    // and 16-byte output stores.
+    const bool allow_split = L->host_kept >= 0 && L->C_out % 8 == 0 && (reinterpret_cast<uintptr_t>(y) & 15) == 0;
+    if (!plan_fast(g, L->num_sms, est_rows, fuse_compact ? (int)L->rows : 0, allow_split, &plan)) return ASX_ERR_UNSUPPORTED;
+    if (plan.ksplit > 1) {
+        const size_t need = (size_t)plan.ws_items * 128 * (size_t)plan.BN * sizeof(float);
+        if (need > L->ws_bytes) {
+            cudaFree(L->d_ws);
+            L->d_ws = nullptr; L->ws_bytes = 0;
+            if (cudaMalloc(&L->d_ws, need) != cudaSuccess) return ASX_ERR_OOM;
+            L->ws_bytes = need;
+        }
+        const size_t ints = 2 * (size_t)(plan.ws_items / plan.ksplit);
+        if (ints > L->wscnt_ints) {
+            cudaFree(L->d_wscnt);
+            L->d_wscnt = nullptr; L->wscnt_ints = 0;
+            if (cudaMalloc(&L->d_wscnt, ints * sizeof(int)) != cudaSuccess) return ASX_ERR_OOM;
+            L->wscnt_ints = ints;
+            if (cudaMemsetAsync(L->d_wscnt, 0, ints * sizeof(int), st) != cudaSuccess) return ASX_ERR_CUDA;
+        }
+    }
     const int Kw = g.K;
     if (L->tmap_ptr != wsrc || L->tmap_BN != plan.BN || L->tmap_Kw != Kw) {
         EncodeTiledFn enc = encode_tiled_fn();
@@ -375,7 +399,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         }
     }
     return from_cuda(launch_fast(g, plan, L->tmap, plan.vec == 2 ? L->tmap_x : L->tmap, xsrc, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
-                                 L->num_sms, fuse_compact ? 1 : 0, L->host_kept, st));
+                                 L->num_sms, fuse_compact ? 1 : 0, L->host_kept, static_cast<float*>(L->d_ws), L->d_wscnt, st));
 }
 
 asx_status asx_get_kept(asx_layer* L, int64_t* count, const int32_t** dev_kept)
@@ -425,6 +449,8 @@ asx_status asx_last_device_status(asx_layer* L)
         cudaMemcpy(&scan_err, static_cast<int32_t*>(L->d_scratch) + 1, sizeof(scan_err), cudaMemcpyDeviceToHost) != cudaSuccess)
         return ASX_ERR_CUDA;
     if (word != 0 && cudaMemset(L->d_small + 1, 0, sizeof(word)) != cudaSuccess) return ASX_ERR_CUDA;
+    // a launch that gave up may have left tile counters of the split-K exchange half way
+    if (word != 0 && L->d_wscnt != nullptr && cudaMemset(L->d_wscnt, 0, L->wscnt_ints * sizeof(int)) != cudaSuccess) return ASX_ERR_CUDA;
     return (word != 0 || scan_err != 0) ? ASX_ERR_TIMEOUT : ASX_OK;
 }
 
@@ -434,7 +460,7 @@ asx_status asx_destroy(asx_layer* L)
     if (L->device >= 0) {
         cudaStreamSynchronize(L->last_stream);
         cudaFree(L->d_mask); cudaFree(L->d_kept); cudaFree(L->d_scratch);
-        cudaFree(L->d_small); cudaFree(L->d_wpack); cudaFree(L->d_xpad);
+        cudaFree(L->d_small); cudaFree(L->d_wpack); cudaFree(L->d_xpad); cudaFree(L->d_ws); cudaFree(L->d_wscnt);
     }
     delete L;
     return ASX_OK;

@@ -40,6 +40,7 @@ constexpr int INFO_RING = 8;            // tiles whose row coordinates are kept 
 constexpr int WARP_ZERO0 = WARP_PROD0 + NUM_PROD_WARPS, NUM_ZERO_WARPS = 4;
 constexpr int WARP_INFO = WARP_ZERO0 + NUM_ZERO_WARPS;
 constexpr int NUM_THREADS = 32 * (WARP_INFO + 1);
+static_assert(NUM_EPI_WARPS * 32 == BM, "one epilogue thread per tile row");
 constexpr long long WAIT_CYCLE_LIMIT = 4000000000ll;   // about two seconds
 
 // Division of a 32-bit unsigned number by a divisor fixed for the whole launch, as a multiply-high
@@ -71,6 +72,7 @@ __device__ __forceinline__ uint32_t fd_div(uint32_t n, const FastDiv& f)
 struct FastArgs {
     FastDiv fdP, fdWo;           // divisions by P and Wo
     FastDiv fdNt;                // division by n_tiles
+    FastDiv fdKs;                // division by ksplit
     FastDiv fdcnt_host;          // division by the kept count when the host knows it (d = 0: it does not)
     const __nv_bfloat16* x;
     const float* bias;
@@ -85,6 +87,10 @@ struct FastArgs {
     int fuse_compact;   // rebuild the kept-row list from the mask inside this kernel (small masks)
     int32_t* kept_out;  // where the fused compaction writes the list and its count
     int32_t* count_out;
+    int ksplit;         // work items per output tile: each takes a contiguous share of the k-blocks
+    float* ws_partial;  // ksplit > 1: [item][128][BN] fp32 partial tiles
+    int* ws_counters;   // ksplit > 1: per output tile {partials written, slices reduced}, zero between launches
+    int ws_items;       // capacity of ws_partial in items
 };
 
 struct alignas(16) Shared {           // lives after the operand stages
@@ -225,6 +231,24 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 
 enum : int { GATHER_CPASYNC = 1, GATHER_TMA = 2 };
 
+// Work item t = (output tile, k share): tile = t / ksplit, share ks = t % ksplit covers k-blocks
+// [ks KB / ksplit, (ks + 1) KB / ksplit).  The shares of a tile are consecutive items, so they run
+// on different blocks at the same time.
+struct Item {
+    int tile, ks, m_tile, n_tile, kb_lo, kb_hi;
+};
+__device__ __forceinline__ Item item_of(int t, int KB, const FastArgs& a)
+{
+    Item it;
+    it.tile = (int)fd_div((uint32_t)t, a.fdKs);
+    it.ks = t - it.tile * a.ksplit;
+    it.m_tile = (int)fd_div((uint32_t)it.tile, a.fdNt);
+    it.n_tile = it.tile - it.m_tile * a.n_tiles;
+    it.kb_lo = it.ks * KB / a.ksplit;
+    it.kb_hi = (it.ks + 1) * KB / a.ksplit;
+    return it;
+}
+
 // What the gather warps need to know about the rk-th kept lowered row: the pixel index of its
 // window's corner, (n H + iy0) W + ix0, and the corner's coordinates packed as iy0 << 16 | ix0.
 // Rows past the end get iy0 = -32768, for which no filter tap is inside the image.
@@ -328,7 +352,11 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     // With every position dropped there are no tiles; the zero warps then write the whole output
     // (Algorithm 2, mask == 0 branch).
     const int m_tiles = (Mk + BM - 1) / BM;
-    const int total_tiles = m_tiles * a.n_tiles;
+    int total_tiles = m_tiles * a.n_tiles * a.ksplit;     // work items
+    if (a.ksplit > 1 && total_tiles > a.ws_items) {       // cannot happen when the host sized the workspace from this mask
+        if (tid == 0) atomicOr(a.dev_status, DEV_BAD_INDEX);
+        total_tiles = 0;
+    }
     FastDiv fdcnt = a.fdcnt_host;
     if (cnt <= 0 || fdcnt.d != (uint32_t)cnt) fdcnt = make_fastdiv((uint32_t)(cnt > 0 ? cnt : 1));   // the host did not know the count
 
@@ -339,7 +367,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             const int jj = idx / BM, rr = idx - jj * BM;
             const long long t = blockIdx.x + (long long)jj * gridDim.x;
             if (t < total_tiles)
-                sh->rowinfo[jj][rr] = row_info_of((int)fd_div((uint32_t)t, a.fdNt) * BM + rr, Mk, fdcnt, g, a, kept_list);
+                sh->rowinfo[jj][rr] = row_info_of(item_of((int)t, KB, a).m_tile * BM + rr, Mk, fdcnt, g, a, kept_list);
         }
         __syncthreads();
         if (tid < INFO_RING && blockIdx.x + (long long)tid * gridDim.x < total_tiles) ptx::mbar_arrive(ptx::smem_u32(&sh->info_full[tid]));
@@ -352,8 +380,9 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             uint32_t ph = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const int n_tile = t - (int)fd_div((uint32_t)t, a.fdNt) * a.n_tiles;
-                for (int kb = 0; kb < KB; ++kb) {
+                const Item item = item_of(t, KB, a);
+                const int n_tile = item.n_tile;
+                for (int kb = item.kb_lo; kb < item.kb_hi; ++kb) {
                     if (!wait_bar<40>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
                     const uint32_t full = ptx::smem_u32(&sh->full[s]);
                     ptx::mbar_arrive_expect_tx(full, (uint32_t)(BN * BK * 2 + (MODE == GATHER_TMA ? A_STAGE_BYTES : 0)));
@@ -377,7 +406,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                 good = wait_bar<200>(ptx::smem_u32(&sh->info_empty[r]), ((uint32_t)(j / INFO_RING) & 1u) ^ 1u, abort_flag, a.dev_status) ? 1 : 0;
             good = __shfl_sync(0xffffffffu, good, 0);
             if (!good) break;
-            const int m_tile = (int)fd_div((uint32_t)t, a.fdNt);
+            const int m_tile = item_of((int)t, KB, a).m_tile;
 #pragma unroll
             for (int q2 = 0; q2 < 4; ++q2) {
                 const int rr = lane * 4 + q2;
@@ -403,7 +432,8 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             if (!ok) break;
             ptx::tc_fence_after_sync();
             const uint32_t d = tmem_base + (uint32_t)(buf * BN);
-            for (int kb = 0; kb < KB; ++kb) {
+            const Item item = item_of(t, KB, a);
+            for (int kb = item.kb_lo; kb < item.kb_hi; ++kb) {
                 ok = warp_wait_bar<0>(ptx::smem_u32(&sh->full[s]), ph, abort_flag, a.dev_status);
                 if (!ok) break;
                 // Only the cp.async gather writes the stage through the generic proxy without a fence
@@ -414,7 +444,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                 const uint64_t adesc = adesc0 + (uint64_t)(s * (stage_bytes >> 4));   // start-address field
                 const uint64_t bdesc = adesc + (A_STAGE_BYTES >> 4);
                 if (ptx::elect_one()) {
-                    ptx::umma_bf16(d, adesc, bdesc, idesc, kb != 0 ? 1u : 0u);       // 16 K-elements = 32 bytes
+                    ptx::umma_bf16(d, adesc, bdesc, idesc, kb != item.kb_lo ? 1u : 0u);       // 16 K-elements = 32 bytes
                     ptx::umma_bf16(d, adesc + 2, bdesc + 2, idesc, 1u);             //   = 2 descriptor units
                     ptx::umma_bf16(d, adesc + 4, bdesc + 4, idesc, 1u);
                     ptx::umma_bf16(d, adesc + 6, bdesc + 6, idesc, 1u);
@@ -433,7 +463,8 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         int ti = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
-            const int m_tile = (int)fd_div((uint32_t)t, a.fdNt), n_tile = t - m_tile * a.n_tiles;
+            const Item item = item_of(t, KB, a);
+            const int m_tile = item.m_tile, n_tile = item.n_tile;
             const int n0 = n_tile * BN;
             // kept rows from the accumulator
             const int buf = ti & 1;
@@ -452,6 +483,109 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             if (!warp_wait_bar<100>(ptx::smem_u32(&sh->acc_full[buf]), use, abort_flag, a.dev_status)) { ok = false; break; }
             ptx::tc_fence_after_sync();
             const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
+            if (a.ksplit > 1) {
+                // ---- split K: this item holds a partial sum.  Every share writes its partial tile
+                // to the workspace; when all shares of the tile are there, each share adds up the
+                // partials of its slice of the tile's rows, always in share order (so the result
+                // does not depend on which block finished first), and writes that slice of y.
+                const int et = (warp - WARP_EPI0) * 32 + lane;
+                // A partial tile is stored as [BN / 4 column groups][128 rows] float4, so that the
+                // warps (one row per lane) write and read whole consecutive lines.
+                float4* mine = reinterpret_cast<float4*>(a.ws_partial) + (size_t)t * (BN >> 2) * BM + (q * 32 + lane);
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t r[32];
+                    if (c0 + 32 <= BN) {
+                        ptx::tmem_ld_32(tacc + (uint32_t)c0, r);
+                    } else {
+                        uint32_t r16[16];
+                        ptx::tmem_ld_16(tacc + (uint32_t)c0, r16);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) { r[j] = r16[j]; r[16 + j] = 0; }
+                    }
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int h = 0; h < 8; ++h)
+                        if (c0 + 4 * h < BN)
+                            __stcg(mine + (size_t)((c0 >> 2) + h) * BM,
+                                   make_float4(__uint_as_float(r[4 * h]), __uint_as_float(r[4 * h + 1]),
+                                               __uint_as_float(r[4 * h + 2]), __uint_as_float(r[4 * h + 3])));
+                }
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[buf]));     // the accumulator is free again
+                int* counters = a.ws_counters + 2 * item.tile;
+                __threadfence();
+                asm volatile("bar.sync 1, %0;" ::"n"(NUM_EPI_WARPS * 32) : "memory");
+                if (et == 0) {
+                    atomicAdd(counters, 1);
+                    const long long t0 = clock64();
+                    while (*reinterpret_cast<volatile int*>(counters) < a.ksplit) {
+                        if (*abort_flag) break;
+                        if (clock64() - t0 > WAIT_CYCLE_LIMIT) {
+                            *abort_flag = 1;
+                            atomicOr(a.dev_status, DEV_TIMEOUT_PIPE);
+                            break;
+                        }
+                        __nanosleep(64);
+                    }
+                    __threadfence();
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(NUM_EPI_WARPS * 32) : "memory");
+                if (*abort_flag) { ok = false; break; }
+                // this share's slice: 8-column groups [g_lo, g_hi) of all 128 rows, one row per lane
+                const int G = BN >> 3;
+                const int g_lo = item.ks * G / a.ksplit, g_hi = (item.ks + 1) * G / a.ksplit;
+                const float4* __restrict__ tile_ws = reinterpret_cast<const float4*>(a.ws_partial) + (size_t)item.tile * a.ksplit * (BN >> 2) * BM;
+                uint4* __restrict__ yv = reinterpret_cast<uint4*>(a.y);
+                const int rk2 = m_tile * BM + et;              // NUM_EPI_WARPS * 32 == BM: thread et owns row et
+                const long long yrow = rk2 < Mk ? (long long)out_row_of(rk2, fdcnt, g, kept_list) * N : -1;
+#pragma unroll 2
+                for (int gq = g_lo; gq < g_hi; ++gq) {
+                    if (yrow < 0 || n0 + gq * 8 >= N) continue;
+                    float4 lo4 = make_float4(0.f, 0.f, 0.f, 0.f), hi4 = lo4;
+                    for (int sp0 = 0; sp0 < a.ksplit; sp0 += 4) {
+                        float4 pl[4], phh[4];
+#pragma unroll
+                        for (int d2 = 0; d2 < 4; ++d2) {
+                            const int sp = sp0 + d2;
+                            if (sp < a.ksplit) {
+                                const float4* src = tile_ws + ((size_t)sp * (BN >> 2) + 2 * gq) * BM + et;
+                                pl[d2] = __ldcg(src);
+                                phh[d2] = __ldcg(src + BM);
+                            } else {
+                                pl[d2] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                phh[d2] = pl[d2];
+                            }
+                        }
+#pragma unroll
+                        for (int d2 = 0; d2 < 4; ++d2) {          // always in share order
+                            lo4.x += pl[d2].x; lo4.y += pl[d2].y; lo4.z += pl[d2].z; lo4.w += pl[d2].w;
+                            hi4.x += phh[d2].x; hi4.y += phh[d2].y; hi4.z += phh[d2].z; hi4.w += phh[d2].w;
+                        }
+                    }
+                    float v[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float f = v[j] + sbias[gq * 8 + j];
+                        v[j] = a.relu ? fmaxf(f, 0.f) : f;
+                    }
+                    uint4 o;
+                    o.x = pack_bf16(v[0], v[1]);
+                    o.y = pack_bf16(v[2], v[3]);
+                    o.z = pack_bf16(v[4], v[5]);
+                    o.w = pack_bf16(v[6], v[7]);
+                    yv[(yrow + n0 + gq * 8) >> 3] = o;
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(NUM_EPI_WARPS * 32) : "memory");
+                if (et == 0) {
+                    // the last share to finish its slice puts the tile's counters back to zero
+                    if (atomicAdd(counters + 1, 1) == a.ksplit - 1) {
+                        atomicExch(counters, 0);
+                        atomicExch(counters + 1, 0);
+                    }
+                }
+                continue;
+            }
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 const int col0 = n0 + c0;
                 if (col0 >= N) break;
@@ -583,8 +717,15 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                     const int pix[4] = {ra.x, ra.z, rb.x, rb.z}, yx[4] = {ra.y, ra.w, rb.y, rb.w};
                     __syncwarp(0xfu);
                     if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));    // the ring slot is in registers now
+                    const Item item = item_of(t, KB, a);
                     int ky = 0, kx = 0, ci = 0;
-                    for (int kb = 0; kb < KB; ++kb, ++it) {
+                    if (item.kb_lo != 0) {                 // a later k share starts inside the window
+                        const int tap = item.kb_lo * BK / g.C_in;
+                        ci = item.kb_lo * BK - tap * g.C_in;
+                        ky = tap / g.kw;
+                        kx = tap - ky * g.kw;
+                    }
+                    for (int kb = item.kb_lo; kb < item.kb_hi; ++kb, ++it) {
                         if ((it & 1) == grp) {
                             const int koff = ky * g.W + kx;
                             int idx[4];
@@ -627,15 +768,16 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));    // the ring slot is in registers now
 
                 // window position (filter tap and channel) of this lane's first K element of the stage
+                const Item item = item_of(t, KB, a);
                 int ky, kx, ci;
                 {
-                    const int k_first = c * 8;
+                    const int k_first = item.kb_lo * BK + c * 8;
                     const int tap = k_first / g.C_in;
                     ci = k_first - tap * g.C_in;
                     ky = tap / g.kw;
                     kx = tap - ky * g.kw;
                 }
-                for (int kb = 0; kb < KB; ++kb, ++it) {
+                for (int kb = item.kb_lo; kb < item.kb_hi; ++kb, ++it) {
                     if ((it & 1) == grp) {
                         if (!warp_wait_bar<40>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
                         const uint32_t stage = smem_base + s * stage_bytes + (uint32_t)(16 * pwg) * 128u;
@@ -722,27 +864,35 @@ __global__ void pack_pair_filters_kernel(const unsigned short* __restrict__ w, u
 
 }  // namespace
 
-bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fused_list_rows, FastPlan* plan)
+bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fused_list_rows, bool allow_split, FastPlan* plan)
 {
     const int N = g.C_out;
     const int KB = (g.K + BK - 1) / BK;
     const long long m_tiles = (est_kept_rows + BM - 1) / BM > 0 ? (est_kept_rows + BM - 1) / BM : 1;
-    // Tile width.  The main loop is bound by shared-memory bandwidth (128 bytes per clock): per
-    // 64-wide k-block the gathered A tile (16 KB) and the filter slab (BN x 128 bytes) are written
-    // once and read once by the tensor core, so a k-block costs about 256 + 2*BN clocks (BN = 64:
-    // 0.20 us, 128: 0.27 us, 256: 0.40 us at 1.9 GHz; measured 0.29 us at 128).  A wider tile does
-    // more work per byte, a narrower one gives more tiles when a layer has few kept rows.  Pick
-    // the width with the lowest estimated time = waves x (k-blocks x time per k-block + fixed).
-    int best_BN = 0;
+    // Tile width and k shares.  A wider tile does more work per gathered byte, a narrower one
+    // gives more tiles when a layer has few kept rows, and sharing a tile's k-blocks between
+    // blocks gives more work items still, at the price of exchanging fp32 partial tiles.  Pick
+    // the pair with the lowest estimated time, from figures measured on B200: a 64-wide k-block
+    // of a 128 x BN tile takes about 0.30 + 0.001 BN microseconds (the loop is bound by the TMA
+    // requests and bytes one SM can pull from L2: 16 KB of gathered rows in 32 requests of about
+    // 13 clocks, plus the BN x 128-byte filter slab), the last tile's epilogue about 0.012 BN,
+    // and the exchange of partial tiles about 7 + 0.025 BN (a chain of write, fence, counter and
+    // read latencies).  Sharing pays where there are far fewer tiles than SMs and K is long.
+    int best_BN = 0, best_KS = 1;
     double best_cost = 0.0;
     for (int n_tiles = (N + 255) / 256; ; n_tiles *= 2) {
         const int per = (N + n_tiles - 1) / n_tiles;
         const int BN = ((per + 15) / 16) * 16;
         const int nt = (N + BN - 1) / BN;
-        const long long waves = (m_tiles * nt + num_sms - 1) / num_sms;
-        const double t_kb = (256.0 + 2.0 * BN) / 1900.0;                    // microseconds
-        const double cost = (double)waves * (KB * t_kb + 2.0);
-        if (best_BN == 0 || cost < best_cost * 0.97) { best_BN = BN; best_cost = cost; }
+        const double t_kb = 0.30 + 0.001 * BN;                                // microseconds
+        for (int KS = 1; KS <= (allow_split ? 8 : 1); ++KS) {
+            if (KS > 1 && KB / KS < 4) break;
+            const long long items = m_tiles * nt * KS;
+            const long long waves = (items + num_sms - 1) / num_sms;
+            const int kbi = (KB + KS - 1) / KS;
+            const double cost = (double)waves * (kbi * t_kb + 0.3) + 0.012 * BN + (KS > 1 ? 7.0 + 0.025 * BN : 0.0);
+            if (best_BN == 0 || cost < best_cost * 0.97) { best_BN = BN; best_KS = KS; best_cost = cost; }
+        }
         if (BN <= 64) break;
     }
     const int BN = best_BN;
@@ -755,6 +905,8 @@ bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fuse
     if (S < MIN_STAGES) return false;
     plan->BN = BN;
     plan->n_tiles = n_tiles;
+    plan->ksplit = best_KS;
+    plan->ws_items = (long long)m_tiles * n_tiles * best_KS;
     plan->stages = S;
     int smem = 1024 + S * stage_bytes + (int)sizeof(Shared) + list_bytes;
     if (smem < 120 * 1024) smem = 120 * 1024;      // one block per SM: tensor memory is not shared out
@@ -768,7 +920,8 @@ bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fuse
 cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorMap& tmap_w,
                         const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
-                        int num_sms, int fuse_compact, long long host_kept, cudaStream_t st)
+                        int num_sms, int fuse_compact, long long host_kept, float* ws_partial, int* ws_counters,
+                        cudaStream_t st)
 {
     FastArgs a;
     a.fdcnt_host = make_fastdiv((uint32_t)(host_kept > 0 && host_kept < (1ll << 31) ? host_kept : 1));
@@ -789,13 +942,18 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     a.fdWo = make_fastdiv((uint32_t)g.Wo);
     a.n_tiles = plan.n_tiles;
     a.fdNt = make_fastdiv((uint32_t)plan.n_tiles);
+    a.ksplit = plan.ksplit;
+    a.fdKs = make_fastdiv((uint32_t)plan.ksplit);
+    a.ws_partial = ws_partial;
+    a.ws_counters = ws_counters;
+    a.ws_items = (int)plan.ws_items;
     a.stages = plan.stages;
     int cols = 32;
     while (cols < 2 * plan.BN) cols <<= 1;
     a.tmem_cols = cols;
     a.vec_out = (g.C_out % 8 == 0 && (reinterpret_cast<uintptr_t>(y) & 15) == 0) ? 1 : 0;
 
-    long long tiles = ((long long)g.M + BM - 1) / BM * plan.n_tiles;
+    long long tiles = ((long long)g.M + BM - 1) / BM * plan.n_tiles * plan.ksplit;
     int grid = (int)(tiles < num_sms ? tiles : num_sms);
     if (grid < 1) grid = 1;
     auto kern = plan.vec == GATHER_TMA ? masked_conv_sm100_kernel<GATHER_TMA> : masked_conv_sm100_kernel<GATHER_CPASYNC>;
