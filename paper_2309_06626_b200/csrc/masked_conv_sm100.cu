@@ -73,6 +73,7 @@ struct FastArgs {
     FastDiv fdP, fdWo;           // divisions by P and Wo
     FastDiv fdNt;                // division by n_tiles
     FastDiv fdKs;                // division by ksplit
+    FastDiv fdCin, fdkw, fdS;    // divisions by C_in, kw and the number of stages (cp.async gather)
     FastDiv fdcnt_host;          // division by the kept count when the host knows it (d = 0: it does not)
     const __nv_bfloat16* x;
     const float* bias;
@@ -240,12 +241,19 @@ struct Item {
 __device__ __forceinline__ Item item_of(int t, int KB, const FastArgs& a)
 {
     Item it;
-    it.tile = (int)fd_div((uint32_t)t, a.fdKs);
-    it.ks = t - it.tile * a.ksplit;
+    if (a.ksplit == 1) {
+        it.tile = t;
+        it.ks = 0;
+        it.kb_lo = 0;
+        it.kb_hi = KB;
+    } else {
+        it.tile = (int)fd_div((uint32_t)t, a.fdKs);
+        it.ks = t - it.tile * a.ksplit;
+        it.kb_lo = (int)fd_div((uint32_t)(it.ks * KB), a.fdKs);
+        it.kb_hi = (int)fd_div((uint32_t)((it.ks + 1) * KB), a.fdKs);
+    }
     it.m_tile = (int)fd_div((uint32_t)it.tile, a.fdNt);
     it.n_tile = it.tile - it.m_tile * a.n_tiles;
-    it.kb_lo = it.ks * KB / a.ksplit;
-    it.kb_hi = (it.ks + 1) * KB / a.ksplit;
     return it;
 }
 
@@ -751,56 +759,61 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         } else {
             const int c = lane & 7;                        // 16-byte chunk of the 128-byte row
             const int rq = lane >> 3;                      // rows 16pwg + rq + {0,4,8,12}
-            int s = 0, j = 0, it = 0;
-            uint32_t ph = 0;
+            // A group owns every second k-block of the whole launch, so its loop steps by two
+            // k-blocks: 128 K elements = adv_tap filter taps and adv_ci channels.
+            const int adv_tap = (2 * BK) / g.C_in, adv_ci = (2 * BK) - adv_tap * g.C_in;
+            // destination of this lane's chunk inside a stage: rows rq, rq + 8 share a swizzle
+            // phase, rows rq + 4, rq + 12 the other
+            const uint32_t dst_a = (uint32_t)((16 * pwg + rq) * 128 + ((c ^ rq) << 4));
+            const uint32_t dst_b = (uint32_t)((16 * pwg + rq + 4) * 128 + ((c ^ (rq + 4)) << 4));
+            int j = 0;
+            uint32_t it0 = 0;                              // k-blocks of the launch before this tile
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++j) {
                 const int r = j & (INFO_RING - 1);
                 if (!warp_wait_bar<100>(ptx::smem_u32(&sh->info_full[r]), (uint32_t)(j / INFO_RING) & 1u, abort_flag, a.dev_status)) break;
                 const int2* info = sh->rowinfo[r] + 16 * pwg;
-                int pix[4], yx[4];
+                int base[4], yx[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int2 ri = info[rq + 4 * i];
-                    pix[i] = ri.x; yx[i] = ri.y;
+                    base[i] = ri.x * g.C_in;               // element offset of the window's corner
+                    yx[i] = ri.y;
                 }
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));    // the ring slot is in registers now
 
-                // window position (filter tap and channel) of this lane's first K element of the stage
                 const Item item = item_of(t, KB, a);
-                int ky, kx, ci;
+                const int kb0 = item.kb_lo + (int)((it0 ^ (uint32_t)grp) & 1u);          // this group's first k-block of the tile
+                // window position (filter tap, channel) of this lane's chunk in k-block kb0
+                int tap, ci;
                 {
-                    const int k_first = item.kb_lo * BK + c * 8;
-                    const int tap = k_first / g.C_in;
+                    const int k_first = kb0 * BK + c * 8;
+                    tap = (int)fd_div((uint32_t)k_first, a.fdCin);
                     ci = k_first - tap * g.C_in;
-                    ky = tap / g.kw;
-                    kx = tap - ky * g.kw;
                 }
-                for (int kb = item.kb_lo; kb < item.kb_hi; ++kb, ++it) {
-                    if ((it & 1) == grp) {
-                        if (!warp_wait_bar<40>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
-                        const uint32_t stage = smem_base + s * stage_bytes + (uint32_t)(16 * pwg) * 128u;
-                        const bool kvalid = ky < g.kh;     // past K: the window is exhausted
-                        const int koff = ky * g.W + kx;
+                uint32_t itk = it0 + (uint32_t)(kb0 - item.kb_lo);
+                for (int kb = kb0; kb < item.kb_hi; kb += 2, itk += 2) {
+                    const int ky = (int)fd_div((uint32_t)tap, a.fdkw), kx = tap - ky * g.kw;
+                    const bool kvalid = ky < g.kh;         // past K: the window is exhausted
+                    const int tapoff = (ky * g.W + kx) * g.C_in + ci;
+                    const uint32_t lap = fd_div(itk, a.fdS);
+                    const int s = (int)(itk - lap * (uint32_t)S);
+                    if (!warp_wait_bar<40>(ptx::smem_u32(&sh->empty[s]), (lap & 1u) ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
+                    const uint32_t stage = smem_base + s * stage_bytes;
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int row = rq + 4 * i;    // (16pwg + row) & 7 == row & 7
-                            const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
-                            const bool in = kvalid && (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
-                            const unsigned short* src = in ? x2 + ((long long)(pix[i] + koff) * g.C_in + ci) : x2;
-                            ptx::cp_async_16(stage + (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)), src, in ? 16u : 0u);
-                        }
-                        ptx::cp_async_mbar_arrive_noinc(ptx::smem_u32(&sh->full[s]));
+                    for (int i = 0; i < 4; ++i) {
+                        const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
+                        const bool in = kvalid && (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
+                        ptx::cp_async_16(stage + ((i & 1) ? dst_b : dst_a) + (uint32_t)((i >> 1) * 1024),
+                                         x2 + (in ? base[i] + tapoff : 0), in ? 16u : 0u);
                     }
-                    // advance the window position by 64 K elements
-                    ci += BK;
-                    while (ci >= g.C_in) {
-                        ci -= g.C_in;
-                        if (++kx == g.kw) { kx = 0; ++ky; }
-                    }
-                    if (++s == S) { s = 0; ph ^= 1u; }
+                    ptx::cp_async_mbar_arrive_noinc(ptx::smem_u32(&sh->full[s]));
+                    tap += adv_tap;
+                    ci += adv_ci;
+                    if (ci >= g.C_in) { ci -= g.C_in; ++tap; }
                 }
+                it0 += (uint32_t)(item.kb_hi - item.kb_lo);
             }
             ptx::cp_async_wait<0>();              // nothing of this thread is in flight at exit
         }
@@ -943,6 +956,9 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     a.n_tiles = plan.n_tiles;
     a.fdNt = make_fastdiv((uint32_t)plan.n_tiles);
     a.ksplit = plan.ksplit;
+    a.fdCin = make_fastdiv((uint32_t)g.C_in);
+    a.fdkw = make_fastdiv((uint32_t)g.kw);
+    a.fdS = make_fastdiv((uint32_t)plan.stages);
     a.fdKs = make_fastdiv((uint32_t)plan.ksplit);
     a.ws_partial = ws_partial;
     a.ws_counters = ws_counters;
