@@ -41,6 +41,7 @@ constexpr int WARP_ZERO0 = WARP_PROD0 + NUM_PROD_WARPS, NUM_ZERO_WARPS = 4;
 constexpr int WARP_INFO = WARP_ZERO0 + NUM_ZERO_WARPS;
 constexpr int NUM_THREADS = 32 * (WARP_INFO + 1);
 static_assert(NUM_EPI_WARPS * 32 == BM, "one epilogue thread per tile row");
+static_assert(NUM_THREADS / 32 < 32, "the fused compaction keeps its running count in slot 31 of the warp totals");
 constexpr long long WAIT_CYCLE_LIMIT = 4000000000ll;   // about two seconds
 
 // Division of a 32-bit unsigned number by a divisor fixed for the whole launch, as a multiply-high
@@ -177,34 +178,43 @@ __device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, i
     int running = 0;
     for (int base = 0; base < rows; base += nthreads * 16) {
         const int first = base + tid * 16;
-        unsigned flags = (base == 0 && early_ok) ? nonzero_bytes16(early) : mask_flags16(mask, rows, first);
-        const int mine = __popc(flags);
-        int incl = mine;
+        const bool wactive = base + warp * 512 < rows;      // warps past the end of the mask only keep the barriers
+        unsigned flags = 0;
+        int mine = 0, incl = 0;
+        if (wactive) {
+            flags = (base == 0 && early_ok) ? nonzero_bytes16(early) : mask_flags16(mask, rows, first);
+            mine = __popc(flags);
+            incl = mine;
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += t;
+            for (int d = 1; d < 32; d <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += t;
+            }
         }
         if (lane == 31) scan_total[warp] = incl;
         __syncthreads();
-        // every warp scans the (at most 32) warp totals with shuffles
-        const int wt = lane < nwarps ? scan_total[lane] : 0;
-        int winc = wt;
+        if (wactive) {
+            // scan of the (at most 27) warp totals with shuffles
+            const int wt = lane < nwarps ? scan_total[lane] : 0;
+            int winc = wt;
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, winc, d);
-            if (lane >= d) winc += t;
+            for (int d = 1; d < 32; d <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, winc, d);
+                if (lane >= d) winc += t;
+            }
+            const int prefix = __shfl_sync(0xffffffffu, winc - wt, warp);
+            const int total = __shfl_sync(0xffffffffu, winc, 31);
+            const int at = running + prefix + incl - mine;
+            if (flags) {
+                // sixteen independent predicated stores instead of a loop over the set bits
+#pragma unroll
+                for (int q2 = 0; q2 < 16; ++q2)
+                    if ((flags >> q2) & 1u) kept_s[at + __popc(flags & ((1u << q2) - 1u))] = (unsigned short)(first + q2);
+            }
+            if (tid == 0) scan_total[31] = running + total;     // slot 31 is no warp's total (27 warps)
         }
-        const int prefix = __shfl_sync(0xffffffffu, winc - wt, warp);
-        const int total = __shfl_sync(0xffffffffu, winc, 31);
-        int at = running + prefix + incl - mine;
-        while (flags) {
-            const int q2 = __ffs(flags) - 1;
-            flags &= flags - 1;
-            kept_s[at++] = (unsigned short)(first + q2);
-        }
-        running += total;
         __syncthreads();
+        running = scan_total[31];
     }
     return running;
 }
