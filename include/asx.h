@@ -110,9 +110,13 @@ asx_status asx_recompact(asx_layer* layer, void* cuda_stream);
  *   y    : device, bf16 [Nb][Ho][Wo][C_out], Ho = (H + 2*pad - kh)/stride + 1 (Wo alike);
  *          16-byte aligned when C_out % 8 == 0, else 2-byte; must not overlap x.
  *   flags: OR of ASX_ACT_RELU, ASX_RECOMPACT, ASX_IMPL_NAIVE.
- * Asynchronous on `cuda_stream`; allocates only when C_in % 8 != 0: the layer then keeps copies of
- * x and w with the channels zero-padded to a multiple of 8 (refreshed by a small kernel on every
- * call), allocated on first use and when they must grow.  Errors: ASX_ERR_NO_MASK, ASX_ERR_SHAPE when
+ * Asynchronous on `cuda_stream`.  Allocates in two cases only, on first use and when the buffers
+ * must grow: when C_in % 8 != 0 the layer keeps copies of x and w with the channels zero-padded to
+ * a multiple of 8 (refreshed by a small kernel on every call); and when a layer has far fewer
+ * 128-row tiles than the GPU has SMs and a long reduction (K of a few thousand), the k range of a
+ * tile is shared between thread blocks that exchange fp32 partial tiles through a layer-owned
+ * workspace (tiles x shares x 128 x tile width floats).  Partial sums are added in a fixed order,
+ * so results do not depend on scheduling.  Errors: ASX_ERR_NO_MASK, ASX_ERR_SHAPE when
  * the mask length is neither Ho*Wo nor Nb*Ho*Wo, ASX_ERR_INVALID_ARG, ASX_ERR_ALIGN,
  * ASX_ERR_UNSUPPORTED when Nb*Ho*Wo or a tensor's element count reaches 2^31.
  */

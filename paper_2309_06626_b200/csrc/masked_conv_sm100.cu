@@ -17,7 +17,10 @@
 //   zero warps      write zeros to the dropped rows of this block's share of the output,
 //                   straight from the mask.  Every output element is written exactly once.
 //
-// The kept-row count is read from device memory, so the host never has to know it.
+// The kept-row list comes from device memory or, for masks of at most 16384 rows, is built by
+// every block in its own shared memory at the start of this kernel (stage i of Section 3.2 fused
+// in); either way the host never has to know the count.  Layers with few kept rows and a long
+// reduction may share a tile's k-blocks between blocks (split K with a fixed-order exchange).
 // All waits are bounded: a wait that runs out sets the status word and every role leaves.
 #include <cuda_bf16.h>
 #include "asx_internal.h"
