@@ -39,6 +39,7 @@ struct asx_layer {
     CUtensorMap tmap_x;                // x as a [pixels][C_in] matrix, for the TMA row gather
     const void* tmapx_ptr = nullptr;
     int64_t tmapx_pixels = 0;
+    int tmapx_stride = 0;              // bytes between rows of the input view
     cudaStream_t last_stream = nullptr;
 };
 
@@ -298,7 +299,59 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     // kernel runs on the padded geometry, the zero channels contribute nothing.
     const void* xsrc = x;
     const void* wsrc = w;
-    if (L->C_in % 8 != 0) {
+    int x_row_stride = 0;              // bytes between rows of the TMA view of the input (0: C_in * 2)
+    // 2x2-block form for the classic network stem (tiny channel count, stride 2, a 7- or 8-wide
+    // filter): pad the channels to 4 and store every aligned 2x2 pixel block as 16 contiguous
+    // values (32 bytes), in a copy with zero borders.  Four horizontally adjacent blocks are then one
+    // contiguous 128-byte run holding two filter rows of a window (8 columns x 2 rows x 4 channels),
+    // i.e. exactly one row of a 64-wide k-block, and consecutive output pixels are consecutive
+    // blocks.  The kernel sees 64 channels per "pixel", ceil((kh + shift) / 2) vertical taps, one
+    // horizontal tap, stride 1 and no padding, and gathers the runs with the TMA row gather through
+    // a view whose rows are 32 bytes apart (rows overlap; the borders make every tap in bounds).
+    // shift = pad & 1 aligns the window to the blocks; the filter gets zero rows / columns there.
+    const int bshift = L->pad & 1;
+    const bool blocks2x2 = L->C_in <= 4 && L->stride == 2 && (W % 2) == 0 && (H % 2) == 0 &&
+                           (L->kw + bshift + 1) / 2 == 4 && L->kh + bshift <= 32;
+    if (blocks2x2) {
+        const int kh2 = (L->kh + bshift + 1) / 2;
+        const int h0 = (L->pad + bshift) / 2;                              // border on the top and left, in blocks
+        const int Hs = (h0 + H / 2 > g.Ho + kh2 - 1) ? h0 + H / 2 : g.Ho + kh2 - 1;
+        const int Ws = (h0 + W / 2 > g.Wo + 3) ? h0 + W / 2 : g.Wo + 3;
+        const int64_t nblocks = (int64_t)Nb * Hs * Ws;
+        if (nblocks * 16 > lim) return ASX_ERR_UNSUPPORTED;
+        const size_t need_x = (size_t)nblocks * 32 + 128, need_w = (size_t)L->C_out * kh2 * 64 * 2;
+        if (need_x > L->xpad_bytes || need_w > L->wpack_bytes) {
+            cudaStreamSynchronize(st);
+            if (need_x > L->xpad_bytes) {
+                cudaFree(L->d_xpad);
+                L->d_xpad = nullptr; L->xpad_bytes = 0;
+                if (cudaMalloc(&L->d_xpad, need_x) != cudaSuccess) return ASX_ERR_OOM;
+                L->xpad_bytes = need_x;
+            }
+            if (need_w > L->wpack_bytes) {
+                cudaFree(L->d_wpack);
+                L->d_wpack = nullptr; L->wpack_bytes = 0;
+                if (cudaMalloc(&L->d_wpack, need_w) != cudaSuccess) return ASX_ERR_OOM;
+                L->wpack_bytes = need_w;
+            }
+            L->tmap_ptr = nullptr;
+            L->tmapx_ptr = nullptr;
+        }
+        cudaError_t e = launch_stage_blocks2x2(x, L->d_xpad, Nb, H, W, L->C_in, Hs, Ws, h0, st);
+        if (e == cudaSuccess) e = launch_pack_block_filters(w, L->d_wpack, L->C_out, L->kh, L->kw, L->C_in, kh2, bshift, st);
+        if (e != cudaSuccess) return from_cuda(e);
+        xsrc = L->d_xpad;
+        wsrc = L->d_wpack;
+        g.C_in = 64;
+        g.kh = kh2;
+        g.kw = 1;
+        g.K = kh2 * 64;
+        g.H = Hs;
+        g.W = Ws;
+        g.stride = 1; g.stride_w = 1;
+        g.pad = 0; g.pad_w = 0;
+        x_row_stride = 32;
+    } else if (L->C_in % 8 != 0) {
         // Pixel-pair form for tiny channel counts under stride 2 (a network's first layer): pad the
         // channels to 4 and read two horizontally adjacent pixels as one 8-channel pixel.  The
         // convolution then has ceil((kw + shift) / 2) horizontal taps, horizontal stride 1 and left
@@ -383,19 +436,20 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         L->tmap_ptr = wsrc; L->tmap_BN = plan.BN; L->tmap_Kw = Kw;
     }
     if (plan.vec == 2) {
-        const int64_t pixels = (int64_t)Nb * H * W;
-        if (L->tmapx_ptr != xsrc || L->tmapx_pixels != pixels) {
+        const int64_t pixels = (int64_t)Nb * g.H * g.W;
+        const int row_stride = x_row_stride ? x_row_stride : g.C_in * 2;
+        if (L->tmapx_ptr != xsrc || L->tmapx_pixels != pixels || L->tmapx_stride != row_stride) {
             EncodeTiledFn enc = encode_tiled_fn();
             if (enc == nullptr) return ASX_ERR_CUDA;
             const cuuint64_t dims[2] = {(cuuint64_t)g.C_in, (cuuint64_t)pixels};
-            const cuuint64_t strides[1] = {(cuuint64_t)g.C_in * 2};
+            const cuuint64_t strides[1] = {(cuuint64_t)row_stride};
             const cuuint32_t box[2] = {64u, 1u};
             const cuuint32_t estr[2] = {1u, 1u};
             const CUresult r = enc(&L->tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(xsrc), dims,
                                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return ASX_ERR_CUDA;
-            L->tmapx_ptr = xsrc; L->tmapx_pixels = pixels;
+            L->tmapx_ptr = xsrc; L->tmapx_pixels = pixels; L->tmapx_stride = row_stride;
         }
     }
     return from_cuda(launch_fast(g, plan, L->tmap, plan.vec == 2 ? L->tmap_x : L->tmap, xsrc, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,

@@ -262,6 +262,9 @@ def iter_small_cases() -> Iterator[LayerSpec]:
         ("t_2x2_c1_s2_p0", 1, 8, 2, 2, 0, 16, 16, 3, 50, 1),
         ("t_4x4_c2_s2_p1", 2, 40, 4, 2, 1, 18, 22, 2, 25, 4),
         ("t_3x3_c4_s1", 4, 16, 3, 1, 1, 14, 15, 2, 50, 1),
+        # stems that take the 2x2-block form: 7-wide with even padding, 8-wide
+        ("t_7x7_c4_s2_p2", 4, 16, 7, 2, 2, 22, 26, 1, 40, 2),
+        ("t_8x8_c2_s2_p2", 2, 24, 8, 2, 2, 20, 24, 2, 30, 1),
         # few rows and a long reduction: the k-blocks of a tile are shared between blocks
         ("t_3x3_c256_n40_longk", 256, 40, 3, 1, 1, 9, 10, 2, 20, 1),
         ("t_3x3_c320_n264_longk", 320, 264, 3, 1, 1, 12, 12, 1, 0, 1),
