@@ -358,15 +358,10 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         cnt = block_compact(a.mask, g.rows, early_mask, early_ok, kept_s, sh->scan_total, NUM_THREADS);
         kept_list.s = kept_s;
     }
-    // From here on the kernel reads what earlier kernels wrote (the kept-row list and its count,
-    // the input) and writes the output and the list, so it waits for them to have finished.
-    ptx::grid_dependency_wait();
-    if (a.fuse_compact) {
-        if (blockIdx.x == 0) {      // the list in global memory, for asx_get_kept and later runs
-            for (int i = tid; i < cnt; i += NUM_THREADS) a.kept_out[i] = (int32_t)kept_s[i];
-            if (tid == 0) *a.count_out = cnt;
-        }
-    } else {
+    // Without the fused compaction the list and its count were written by an earlier kernel: wait
+    // for it here.  With it, the wait comes after the row decoding below, which needs only the list.
+    if (!a.fuse_compact) {
+        ptx::grid_dependency_wait();
         cnt = *a.count;
     }
     const int Mk = (g.rows == g.P) ? g.Nb * cnt : cnt;
@@ -392,6 +387,15 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         }
         __syncthreads();
         if (tid < INFO_RING && blockIdx.x + (long long)tid * gridDim.x < total_tiles) ptx::mbar_arrive(ptx::smem_u32(&sh->info_full[tid]));
+    }
+    // From here on the kernel reads what earlier kernels wrote (the input, the filters) and writes
+    // the output and the list, so it waits for them to have finished.
+    if (a.fuse_compact) {
+        ptx::grid_dependency_wait();
+        if (blockIdx.x == 0) {      // the list in global memory, for asx_get_kept and later runs
+            for (int i = tid; i < cnt; i += NUM_THREADS) a.kept_out[i] = (int32_t)kept_s[i];
+            if (tid == 0) *a.count_out = cnt;
+        }
     }
 
     if (warp == WARP_TMA) {
