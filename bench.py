@@ -37,12 +37,12 @@ L2_BYTES = 126 * 1024 * 1024
 
 # DRAM traffic of the dominant kernel from one ncu capture of the default workload (ResNet-18 stack,
 # batch 64): dram__bytes_read.sum + dram__bytes_write.sum averaged over the 20 fused-kernel launches
-# of a step (12.11 MB read + 2.35 MB written; ncu flushes the caches before every captured launch,
+# of a step (12.18 MB read + 2.35 MB written; ncu flushes the caches before every captured launch,
 # so reads are cold-cache and most of a launch's output is still in L2 when its counters stop).
 # The figure belongs to the kernel sources whose digest is recorded with it; with any other sources
 # the bench reports null.
-NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.47e6,
-               "csrc_sha256": "90ecd06c7a308f7155f533f6b06f81ff58da77a7a982d4f7178539b53ae39a9b"}
+NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.52e6,
+               "csrc_sha256": "b272c8b853797078760592fadeaab1aa386cc531f824fad201f2ffa0d9e9d7cc"}
 
 
 def csrc_digest() -> str:
