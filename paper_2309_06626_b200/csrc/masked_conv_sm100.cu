@@ -907,6 +907,24 @@ __global__ void stage_blocks2x2_kernel(const unsigned short* __restrict__ x, uin
         const long long rest = i / Ws;
         const int by = (int)(rest % Hs), n = (int)(rest / Hs);
         unsigned short v[16];
+        if (C == 3 && (reinterpret_cast<uintptr_t>(x) & 3) == 0) {
+            // three channels: the two pixels of a block row are 12 contiguous bytes at a 4-byte
+            // aligned offset (the block's first column is even), i.e. three 32-bit loads
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int iy = 2 * (by - h0) + r, ix = 2 * (bx - h0);
+                const bool in = iy >= 0 && iy < H && ix >= 0 && ix < W;       // W is even: both pixels or none
+                uint32_t q0 = 0, q1 = 0, q2 = 0;
+                if (in) {
+                    const uint32_t* src = reinterpret_cast<const uint32_t*>(x + (((long long)n * H + iy) * W + ix) * 3);
+                    q0 = __ldg(src); q1 = __ldg(src + 1); q2 = __ldg(src + 2);
+                }
+                v[r * 8 + 0] = (unsigned short)(q0 & 0xffffu); v[r * 8 + 1] = (unsigned short)(q0 >> 16);
+                v[r * 8 + 2] = (unsigned short)(q1 & 0xffffu); v[r * 8 + 3] = 0;
+                v[r * 8 + 4] = (unsigned short)(q1 >> 16);     v[r * 8 + 5] = (unsigned short)(q2 & 0xffffu);
+                v[r * 8 + 6] = (unsigned short)(q2 >> 16);     v[r * 8 + 7] = 0;
+            }
+        } else
 #pragma unroll
         for (int r = 0; r < 2; ++r)
 #pragma unroll

@@ -11,7 +11,7 @@ import torch
 import oracle
 import paper_2309_06626_b200 as asx
 import workloads as wl
-from gpu_util import check_against_oracle, make_problem, run_library
+from gpu_util import check_against_oracle, make_problem, run_library, to_dev_bf16
 from philox_ref import random_block_mask
 
 pytestmark = pytest.mark.gpu
@@ -124,3 +124,25 @@ def test_config1_full():
     x, w, b, mask = make_problem(spec)
     assert int(mask.sum()) == 1568
     check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU)
+
+
+def test_shared_k_blocks_give_the_same_bits_every_run():
+    """Few kept rows and a long reduction: the k-blocks of a tile are shared between thread blocks
+    that exchange fp32 partial tiles.  The partials are added in a fixed order, so repeated runs
+    (and a run on the same layer handle after the workspace was used) agree bit for bit."""
+    spec = [s for s in SMALL if s.name == "t_3x3_c512"][0]
+    x, w, b, mask = make_problem(spec)
+    layer = asx.MaskedConvLayer(spec.C_in, spec.C_out, spec.kh, spec.kw, spec.stride, spec.pad)
+    layer.set_mask(mask)
+    xd, wd, bd = to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda()
+    runs = []
+    for flags in (asx.ACT_RELU, asx.ACT_RELU | asx.RECOMPACT, asx.ACT_RELU):
+        y = layer.run(xd, wd, bd, flags=flags)
+        torch.cuda.synchronize()
+        runs.append(y.view(torch.int16).cpu().numpy().copy())
+    assert layer.device_status() == 0
+    layer.close()
+    assert np.array_equal(runs[0], runs[1]) and np.array_equal(runs[0], runs[2])
+    ref = oracle.masked_conv(x, w, b, mask, spec.stride, spec.pad, True)
+    got = torch.from_numpy(runs[0]).view(torch.bfloat16).float().numpy().astype(np.float64).reshape(ref.shape)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) < 5e-3
