@@ -42,7 +42,7 @@ L2_BYTES = 126 * 1024 * 1024
 # The figure belongs to the kernel sources whose digest is recorded with it; with any other sources
 # the bench reports null.
 NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.52e6,
-               "csrc_sha256": "580a9f36bad5662a323a30a35498aa9e2981ba1667d831c8de0b39f1577867e2"}
+               "csrc_sha256": "ebb65e8abacbcb5a99906144289768774d0f87f5a801ecf3b2e5f82161788506"}
 
 
 def csrc_digest() -> str:
@@ -208,10 +208,12 @@ def run_reference(args):
 # --------------------------------------------------------------------------------------------
 # the GPU leg
 class DeviceLayer:
-    def __init__(self, spec, torch, asx, dense_twin=True):
+    def __init__(self, spec, torch, asx, dense_twin=True, score=None):
         self.spec = spec
         x, w, b = wl.make_x(spec), wl.make_w(spec), wl.make_b(spec)
-        self.mask = wl.make_layer_mask(spec)
+        # masks: seeded blocks of rows (default), or the paper's generator from one input-resolution score
+        self.mask = (wl.make_layer_mask(spec) if score is None
+                     else asx.mask_from_scores(score, spec.Ho, spec.Wo, spec.sparsity_pct / 100.0))
         self.x_host = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
         self.x = self.x_host.cuda()
         self.w = torch.from_numpy(w).to(torch.bfloat16).cuda()
@@ -272,7 +274,10 @@ def run_ours(args):
         specs = [s for s in specs if any(s.name.startswith(p) for p in args.only.split(","))]
         if not specs:
             raise SystemExit(f"--only {args.only}: no such layer")
-    layers = [DeviceLayer(s, torch, asx, dense_twin=(args.config != 5)) for s in specs]
+    score = None
+    if args.mask == "scores":
+        score = wl.make_score(args.config, max(s.H for s in specs), max(s.W for s in specs))
+    layers = [DeviceLayer(s, torch, asx, dense_twin=(args.config != 5), score=score) for s in specs]
     torch.cuda.synchronize()
     footprint = sum(L.x.numel() * 2 + L.y.numel() * 2 + L.w.numel() * 2 for L in layers)
 
@@ -475,7 +480,9 @@ def run_ours(args):
                    "step": "per layer: one asx_run with ASX_RECOMPACT = mask compaction (inside the fused kernel "
                            "for masks <= 16384 rows) + gather/GEMM/scatter"
                            + ("" if graph is None else "; one step = one CUDA-graph replay"),
-                   "mask": "one mask per layer shared by the batch"},
+                   "mask": "one mask per layer shared by the batch"
+                           + ("" if args.mask == "blocks" else "; masks from one random input-resolution score, average-pooled"
+                              " to each layer and ranked (Algorithm 1, getMask)")},
         "dense_equivalent_tflops": world * dense_flops_step / (ms_step * 1e-3) / 1e12,
         "speedup_vs_sparsity0": (ms_dense / ms_step) if args.config != 5 else None,
         "ms_per_step_sparsity0": ms_dense,
@@ -486,7 +493,7 @@ def run_ours(args):
                 "ms_per_step": e2e_ms},
         "gpu_launches": K * sum(L.launches for L in layers),
         "roofline": {"bound": "tensor", "kernel": "masked_conv_sm100_kernel", "achieved": achieved,
-                     "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": measured_traffic(args.config, args.only),
+                     "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": measured_traffic(args.config, args.only or (args.mask != "blocks")),
                      "traffic_unit": "bytes per launch (ncu dram read + write, average over the step's fused-kernel launches)",
                      "algorithmic_bytes_per_launch": sum(L.bytes for L in layers) / len(layers),
                      "peak_source": f"{peaks['source']} (sustained bf16 matmul; burst {peaks['bf16_tflops']})",
@@ -513,6 +520,8 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--mask", default="blocks", choices=["blocks", "scores"],
+                    help="blocks: seeded blocks of dropped rows; scores: the paper's getMask from one random score")
     ap.add_argument("--no-s1", action="store_true", help="skip the stand-alone compaction bandwidth leg")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

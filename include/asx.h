@@ -94,6 +94,27 @@ asx_status asx_set_mask_random(asx_layer* layer, int64_t rows, double sparsity, 
                                uint64_t seed, void* cuda_stream);
 
 /*
+ * The mask generator of the paper's training pipeline (Algorithm 1, function getMask) for one layer:
+ * a 2-D score at the input image's resolution is brought to the layer's resolution by an average
+ * pooling with window = stride = ratio, ratio = input_res // layer_res per axis, the layer's
+ * positions are ranked by their pooled score, and the mask is 0 at the ranked fraction `sparsity`.
+ * Using one score for all layers of a network gives masks that agree across resolutions
+ * (Section 3.1).  Where the paper is silent this library takes: the floor(sparsity*P + 1/2)
+ * positions with the SMALLEST pooled score are dropped (P = Ho*Wo); equal scores are ordered by
+ * position (raster order); output cell (i, j) pools score rows i*rh .. i*rh+rh-1 and columns
+ * j*rw .. j*rw+rw-1 with rh = H0 / Ho, rw = W0 / Wo (integer division; what lies beyond is unused);
+ * window sums are accumulated in fp64 in raster order and divided by rh*rw in fp64.
+ *   score    : HOST pointer, H0*W0 floats, row-major.  1 <= Ho <= H0, 1 <= Wo <= W0, 0 <= sparsity <= 1.
+ *   mask_out : HOST pointer, receives Ho*Wo bytes (1 keep / 0 drop).
+ * asx_mask_from_scores runs on the host only (no CUDA call); asx_set_mask_from_scores generates the
+ * mask and sets it like asx_set_mask (mask shared by the batch).
+ */
+asx_status asx_mask_from_scores(const float* score, int H0, int W0, int Ho, int Wo, double sparsity,
+                                uint8_t* mask_out);
+asx_status asx_set_mask_from_scores(asx_layer* layer, const float* score, int H0, int W0, int Ho, int Wo,
+                                    double sparsity, void* cuda_stream);
+
+/*
  * Rebuild the kept-row list from the stored mask (stage i alone; the same work the
  * ASX_RECOMPACT flag does inside asx_run).  Asynchronous on `cuda_stream`; allocates nothing.
  * ASX_ERR_NO_MASK before any asx_set_mask*.

@@ -16,6 +16,7 @@ EXPORTS = (
     "asx_status_string", "asx_create_layer", "asx_set_mask", "asx_set_mask_random", "asx_recompact", "asx_run",
     "asx_get_kept", "asx_get_kept_host", "asx_get_mask", "asx_last_device_status", "asx_destroy",
     "asx_compact_scratch_bytes", "asx_compact", "asx_compact_status", "asx_compact_static",
+    "asx_mask_from_scores", "asx_set_mask_from_scores",
 )
 COMPACT_STATIC_MAX_ROWS = 1 << 24
 
@@ -57,6 +58,8 @@ def lib():
         L.asx_compact.argtypes = [vp, i64, vp, vp, vp, i64, vp]
         L.asx_compact_status.argtypes = [vp, vp]
         L.asx_compact_static.argtypes = [vp, i64, vp, vp, vp]
+        L.asx_mask_from_scores.argtypes = [vp, ci, ci, ci, ci, ctypes.c_double, vp]
+        L.asx_set_mask_from_scores.argtypes = [vp, vp, ci, ci, ci, ci, ctypes.c_double, vp]
         for name in EXPORTS:
             if name not in ("asx_status_string", "asx_compact_scratch_bytes"):
                 getattr(L, name).restype = ci
@@ -105,6 +108,13 @@ class MaskedConvLayer:
     def set_mask_random(self, rows: int, sparsity: float, block: int, seed: int, stream=None) -> None:
         _check(lib().asx_set_mask_random(self._h, rows, float(sparsity), block, seed, _stream_ptr(stream)),
                "asx_set_mask_random")
+
+    def set_mask_from_scores(self, score, Ho: int, Wo: int, sparsity: float, stream=None) -> None:
+        """Mask of Algorithm 1's getMask for this layer from a host fp32 score map [H0][W0]."""
+        import numpy as np
+        sc = np.ascontiguousarray(score, dtype=np.float32)
+        _check(lib().asx_set_mask_from_scores(self._h, sc.ctypes.data, sc.shape[0], sc.shape[1], Ho, Wo,
+                                              float(sparsity), _stream_ptr(stream)), "asx_set_mask_from_scores")
 
     def recompact(self, stream=None) -> None:
         _check(lib().asx_recompact(self._h, _stream_ptr(stream)), "asx_recompact")
@@ -172,6 +182,16 @@ class MaskedConvLayer:
             self.close()
         except Exception:
             pass
+
+
+def mask_from_scores(score, Ho: int, Wo: int, sparsity: float):
+    """Algorithm 1's getMask for one layer on the host: numpy uint8 [Ho*Wo] from a fp32 score map."""
+    import numpy as np
+    sc = np.ascontiguousarray(score, dtype=np.float32)
+    out = np.empty(Ho * Wo, dtype=np.uint8)
+    _check(lib().asx_mask_from_scores(sc.ctypes.data, sc.shape[0], sc.shape[1], Ho, Wo, float(sparsity),
+                                      out.ctypes.data), "asx_mask_from_scores")
+    return out
 
 
 def compact_mask(mask_dev, stream=None):

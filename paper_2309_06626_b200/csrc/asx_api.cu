@@ -5,6 +5,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <cmath>
 #include <vector>
 
 #include "asx_internal.h"
@@ -228,6 +229,53 @@ asx_status asx_set_mask_random(asx_layer* L, int64_t rows, double sparsity, int 
         std::memset(mask.data() + lo, 0, (size_t)(hi - lo));
     }
     return asx_set_mask(L, mask.data(), rows, cuda_stream);
+}
+
+asx_status asx_mask_from_scores(const float* score, int H0, int W0, int Ho, int Wo, double sparsity,
+                                uint8_t* mask_out)
+{
+    if (score == nullptr || mask_out == nullptr || H0 < 1 || W0 < 1 || Ho < 1 || Wo < 1 || Ho > H0 || Wo > W0 ||
+        !(sparsity >= 0.0 && sparsity <= 1.0) || (int64_t)Ho * Wo >= (1ll << 31))
+        return ASX_ERR_INVALID_ARG;
+    const int rh = H0 / Ho, rw = W0 / Wo;                 // ratio = input_res // layer.res
+    const int64_t P = (int64_t)Ho * Wo;
+    std::vector<std::pair<double, int64_t>> ranked;       // (pooled score, position): ordered by score, then position
+    try {
+        ranked.resize((size_t)P);
+    } catch (const std::bad_alloc&) {
+        return ASX_ERR_OOM;
+    }
+    for (int i = 0; i < Ho; ++i)
+        for (int j = 0; j < Wo; ++j) {
+            double acc = 0.0;                              // window sum in fp64, raster order of the window
+            const float* win = score + (size_t)i * rh * W0 + (size_t)j * rw;
+            for (int a2 = 0; a2 < rh; ++a2)
+                for (int b2 = 0; b2 < rw; ++b2) acc += (double)win[(size_t)a2 * W0 + b2];
+            const int64_t p = (int64_t)i * Wo + j;
+            ranked[(size_t)p] = {acc / (double)(rh * rw), p};
+        }
+    int64_t n_drop = (int64_t)std::floor(sparsity * (double)P + 0.5);
+    if (n_drop > P) n_drop = P;
+    if (n_drop > 0 && n_drop < P) std::nth_element(ranked.begin(), ranked.begin() + (n_drop - 1), ranked.end());
+    std::memset(mask_out, 1, (size_t)P);
+    for (int64_t k = 0; k < n_drop; ++k) mask_out[(size_t)ranked[(size_t)k].second] = 0;
+    return ASX_OK;
+}
+
+asx_status asx_set_mask_from_scores(asx_layer* L, const float* score, int H0, int W0, int Ho, int Wo,
+                                    double sparsity, void* cuda_stream)
+{
+    if (L == nullptr) return ASX_ERR_INVALID_ARG;
+    if (Ho < 1 || Wo < 1) return ASX_ERR_INVALID_ARG;
+    std::vector<uint8_t> mask;
+    try {
+        mask.resize((size_t)Ho * (size_t)Wo);
+    } catch (const std::bad_alloc&) {
+        return ASX_ERR_OOM;
+    }
+    const asx_status s = asx_mask_from_scores(score, H0, W0, Ho, Wo, sparsity, mask.data());
+    if (s != ASX_OK) return s;
+    return asx_set_mask(L, mask.data(), (int64_t)Ho * Wo, cuda_stream);
 }
 
 asx_status asx_recompact(asx_layer* L, void* cuda_stream)

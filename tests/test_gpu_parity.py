@@ -146,3 +146,29 @@ def test_shared_k_blocks_give_the_same_bits_every_run():
     ref = oracle.masked_conv(x, w, b, mask, spec.stride, spec.pad, True)
     got = torch.from_numpy(runs[0]).view(torch.bfloat16).float().numpy().astype(np.float64).reshape(ref.shape)
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) < 5e-3
+
+
+def test_masks_from_one_score_across_resolutions():
+    """Algorithm 1's getMask through the layer API: three layers at different resolutions take their
+    masks from one input-resolution score; the stored masks equal the oracle's bit for bit and the
+    convolutions under them match the oracle."""
+    rng = np.random.default_rng(2309)
+    score = rng.random((32, 48)).astype(np.float32)
+    for (cin, cout, k, s, p, H, W, sparsity) in [(3, 16, 3, 2, 1, 32, 48, 0.3), (16, 32, 3, 1, 1, 16, 24, 0.5),
+                                                 (64, 64, 1, 2, 0, 16, 24, 0.25)]:
+        spec = wl.LayerSpec("scores", cin, cout, k, k, s, p, H, W, 2, int(sparsity * 100), 1, "relu", wl.BASE_SEED + 77)
+        x, w, b = wl.make_x(spec), wl.make_w(spec), wl.make_b(spec)
+        want = oracle.get_mask(score, spec.Ho, spec.Wo, sparsity)
+        layer = asx.MaskedConvLayer(cin, cout, k, k, s, p)
+        layer.set_mask_from_scores(score, spec.Ho, spec.Wo, sparsity)
+        assert np.array_equal(layer.mask(spec.P), want)
+        y = layer.run(to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda(), flags=asx.ACT_RELU | asx.RECOMPACT)
+        torch.cuda.synchronize()
+        assert layer.device_status() == 0
+        assert np.array_equal(layer.kept(), oracle.kept_list(want))
+        layer.close()
+        ref = oracle.masked_conv(x, w, b, want, s, p, True)
+        got = y.float().cpu().numpy().astype(np.float64).reshape(ref.shape)
+        assert np.linalg.norm(got - ref) / np.linalg.norm(ref) < 5e-3
+        dropped = np.tile(want, spec.Nb) == 0
+        assert not got.reshape(spec.M, cout)[dropped].any()

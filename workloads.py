@@ -231,6 +231,13 @@ def algorithmic_flops(spec: LayerSpec, kept_rows: int) -> int:
     return 2 * kept_rows * spec.K * spec.N
 
 
+def make_score(cfg: int, H0: int, W0: int) -> np.ndarray:
+    """The random 2-D score of Algorithm 1's getMask at the network's input resolution: uniform
+    fp32 in [0, 1), one per configuration (every layer of the stack derives its mask from it)."""
+    rng = np.random.Generator(np.random.PCG64(BASE_SEED + 500_000 + cfg))
+    return rng.random((H0, W0), dtype=np.float32)
+
+
 def algorithmic_bytes(spec: LayerSpec, mask: np.ndarray) -> int:
     """Bytes the method must move for one layer call: touched input pixels, weights,
     bias, the full output (zero rows included), the mask and the kept-row list."""
