@@ -5,7 +5,7 @@ It shares no code with the CUDA path and never imports it.
 """
 from .masked_conv import (build, bf16_round, kept_list, masked_conv, masked_conv_rows,
                           n_threads)
-from .get_mask import get_mask, pooled_score
+from .get_mask import get_mask, mask_from_activation, pooled_score
 
 __all__ = ["build", "bf16_round", "kept_list", "masked_conv", "masked_conv_rows", "n_threads",
-           "get_mask", "pooled_score"]
+           "get_mask", "mask_from_activation", "pooled_score"]

@@ -50,3 +50,22 @@ def get_mask(score: np.ndarray, Ho: int, Wo: int, sparsity: float) -> np.ndarray
     for p in order[:k]:
         mask[p] = 0
     return mask
+
+
+def mask_from_activation(x: np.ndarray) -> np.ndarray:
+    """Data-dependent mask of the family the paper contrasts itself with (Section 2: sparsity that
+    comes from the activations themselves, e.g. ReLU zeros): a lowered row / spatial position is kept
+    iff at least one of its channels is strictly positive.  x: [..., C] real values (already rounded
+    to the storage precision by the caller); NaN and zeros of either sign count as not positive.
+    Returns uint8 [prod(leading dims)]."""
+    x = np.asarray(x, dtype=np.float64)
+    C = x.shape[-1]
+    rows = x.reshape(-1, C)
+    out = np.zeros(rows.shape[0], dtype=np.uint8)
+    for r in range(rows.shape[0]):
+        keep = 0
+        for c in range(C):
+            if rows[r, c] > 0.0:
+                keep = 1
+        out[r] = keep
+    return out

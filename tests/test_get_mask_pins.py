@@ -84,3 +84,21 @@ def test_masks_of_two_layers_come_from_the_same_score():
     assert np.argwhere(coarse == 0).tolist() == [[1, 2]]
     np.testing.assert_allclose(oracle.pooled_score(score, 4, 4),
                                oracle.pooled_score(score, 8, 8).reshape(4, 2, 4, 2).mean(axis=(1, 3)), rtol=1e-14)
+
+
+def test_mask_from_activation_special_values_and_library_reduction():
+    x = np.zeros((9, 4), dtype=np.float32)
+    x[1, 2] = 1.0                                   # one positive channel
+    x[2, :] = -1.0                                  # only negatives
+    x[3, 0] = -0.0
+    x[4, 1] = np.nan                                # NaN is not positive
+    x[5, 3] = np.float32(1e-40)                     # a denormal is positive
+    x[6, :] = [np.nan, -1.0, 0.0, 2.0]              # NaN beside a positive
+    x[7, 0] = np.inf
+    x[8, 0] = -np.inf
+    assert oracle.mask_from_activation(x).tolist() == [0, 1, 0, 0, 0, 1, 1, 1, 0]
+    rng = np.random.default_rng(11)
+    y = rng.standard_normal((3, 5, 7, 6)).astype(np.float32)
+    y[rng.random(y.shape[:-1]) < 0.4] = -np.abs(y[rng.random(y.shape[:-1]) < 0.4][0])   # many all-negative positions
+    ref = (torch.from_numpy(y) > 0).any(dim=-1).reshape(-1).numpy().astype(np.uint8)
+    assert np.array_equal(oracle.mask_from_activation(y), ref)
