@@ -42,7 +42,7 @@ L2_BYTES = 126 * 1024 * 1024
 # The figure belongs to the kernel sources whose digest is recorded with it; with any other sources
 # the bench reports null.
 NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.52e6,
-               "csrc_sha256": "ebb65e8abacbcb5a99906144289768774d0f87f5a801ecf3b2e5f82161788506"}
+               "csrc_sha256": "ca50148a1614768f034ac4cf1e63dee4f6aed96c626523ef405670b033ff32dd"}
 
 
 def csrc_digest() -> str:
@@ -460,6 +460,34 @@ def run_ours(args):
               "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "peak_gbs": peaks["hbm_gbs"]}
         del big, kept_big, scr
 
+    # ---- the data-dependent mask kernel alone (HBM-bound: rows*C*2 bytes read, rows written)
+    mfa = None
+    if not args.no_s1:
+        rows_a, C_a = 1 << 22, 64                                   # 512 MB of bf16 activations, larger than L2
+        act = torch.randn((rows_a, C_a), device="cuda", dtype=torch.bfloat16).relu_()
+        act[::3] = 0
+        mask_a = torch.empty(rows_a, dtype=torch.uint8, device="cuda")
+
+        def mfa_call():
+            rc = asx.lib().asx_mask_from_activation(act.data_ptr(), rows_a, C_a, mask_a.data_ptr(), st)
+            if rc:
+                raise RuntimeError(f"asx_mask_from_activation failed with status {rc}")
+        for _ in range(3):
+            mfa_call()
+        torch.cuda.synchronize()
+        m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        m0.record(st_obj)
+        for _ in range(10):
+            mfa_call()
+        m1.record(st_obj)
+        torch.cuda.synchronize()
+        ms_a = m0.elapsed_time(m1) / 10
+        gbs_a = (rows_a * C_a * 2 + rows_a) / (ms_a * 1e-3) / 1e9
+        mfa = {"rows": rows_a, "C": C_a, "ms": ms_a, "gbs": gbs_a, "bytes": "rows*C*2 read + rows written",
+               "frac_of_hbm_peak": gbs_a / peaks["hbm_gbs"], "peak_gbs": peaks["hbm_gbs"],
+               "kept": int(mask_a.sum().item())}
+        del act, mask_a
+
     sweep = None
     if args.config == 5:
         base = {L.spec.block: per_layer_ms[i] for i, L in enumerate(layers) if L.spec.sparsity_pct == 0}
@@ -502,6 +530,7 @@ def run_ours(args):
                      "layer_roofs_ms_per_step": roof_ms},
         "cpu_baseline": cpu,
         "s1_compaction": s1,
+        "mask_from_activation": mfa,
         "sweep": sweep,
         "per_layer": [{"name": L.spec.name, "M": L.spec.M, "K": L.spec.K, "N": L.spec.N, "kept_rows": L.kept_rows,
                        "ms": per_layer_ms[i], "tflops": L.flops / (per_layer_ms[i] * 1e-3) / 1e12,

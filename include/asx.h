@@ -191,6 +191,20 @@ asx_status asx_compact(const uint8_t* mask_dev, int64_t rows, int32_t* kept_dev,
 asx_status asx_compact_status(const void* scratch_dev, void* cuda_stream);
 
 /*
+ * Data-dependent mask (the family the paper contrasts its fixed masks with in Section 2: sparsity
+ * that comes from the activations themselves, such as the zeros a ReLU leaves): mask_dev[r] = 1 iff
+ * at least one of the C channels of row r of a bfloat16 tensor [rows][C] is strictly positive
+ * (zeros of either sign and NaN are not positive; denormals and +inf are).  The result has one
+ * entry per lowered row and can be given to asx_set_mask as a device pointer (rows = Nb*Ho*Wo),
+ * followed by asx_run with ASX_RECOMPACT or not.
+ *   x_dev    : device, bf16 [rows][C], 2-byte aligned (16-byte aligned input with C in
+ *              {8, 16, 32, 64, 128, 256} takes the vectorised kernel).
+ *   mask_dev : device, `rows` bytes, written 0 / 1.   0 <= rows < 2^31, 1 <= C <= 2^20.
+ * Asynchronous on `cuda_stream`; allocates nothing.
+ */
+asx_status asx_mask_from_activation(const void* x_dev, int64_t rows, int C, uint8_t* mask_dev, void* cuda_stream);
+
+/*
  * Mask compaction without any allocation (the paper has no counterpart: this is a convenience
  * of this library).  Same inputs, outputs and result as asx_compact, but the scan's scratch is
  * a fixed array inside the library, so neither the caller nor the library allocates anything:

@@ -5,8 +5,8 @@ CUDA stream); every step of the path runs in the library's CUDA kernels.  Import
 package does not load the library; the first call does, and fails loudly if the library
 has not been built.
 """
-from .binding import (AsxError, MaskedConvLayer, compact_mask, mask_from_scores, lib, lib_path, EXPORTS,
+from .binding import (AsxError, MaskedConvLayer, compact_mask, mask_from_scores, mask_from_activation, lib, lib_path, EXPORTS,
                       ACT_RELU, RECOMPACT, IMPL_NAIVE)
 
-__all__ = ["AsxError", "MaskedConvLayer", "compact_mask", "mask_from_scores", "lib", "lib_path", "EXPORTS",
+__all__ = ["AsxError", "MaskedConvLayer", "compact_mask", "mask_from_scores", "mask_from_activation", "lib", "lib_path", "EXPORTS",
            "ACT_RELU", "RECOMPACT", "IMPL_NAIVE"]

@@ -16,7 +16,7 @@ EXPORTS = (
     "asx_status_string", "asx_create_layer", "asx_set_mask", "asx_set_mask_random", "asx_recompact", "asx_run",
     "asx_get_kept", "asx_get_kept_host", "asx_get_mask", "asx_last_device_status", "asx_destroy",
     "asx_compact_scratch_bytes", "asx_compact", "asx_compact_status", "asx_compact_static",
-    "asx_mask_from_scores", "asx_set_mask_from_scores",
+    "asx_mask_from_scores", "asx_set_mask_from_scores", "asx_mask_from_activation",
 )
 COMPACT_STATIC_MAX_ROWS = 1 << 24
 
@@ -58,6 +58,7 @@ def lib():
         L.asx_compact.argtypes = [vp, i64, vp, vp, vp, i64, vp]
         L.asx_compact_status.argtypes = [vp, vp]
         L.asx_compact_static.argtypes = [vp, i64, vp, vp, vp]
+        L.asx_mask_from_activation.argtypes = [vp, i64, ci, vp, vp]
         L.asx_mask_from_scores.argtypes = [vp, ci, ci, ci, ci, ctypes.c_double, vp]
         L.asx_set_mask_from_scores.argtypes = [vp, vp, ci, ci, ci, ci, ctypes.c_double, vp]
         for name in EXPORTS:
@@ -191,6 +192,20 @@ def mask_from_scores(score, Ho: int, Wo: int, sparsity: float):
     out = np.empty(Ho * Wo, dtype=np.uint8)
     _check(lib().asx_mask_from_scores(sc.ctypes.data, sc.shape[0], sc.shape[1], Ho, Wo, float(sparsity),
                                       out.ctypes.data), "asx_mask_from_scores")
+    return out
+
+
+def mask_from_activation(x_dev, stream=None):
+    """mask[r] = 1 iff a channel of row r of the CUDA bf16 tensor x_dev [..., C] is positive; returns a
+    CUDA uint8 tensor with one entry per row (allocated by torch)."""
+    import torch
+    if x_dev.dtype != torch.bfloat16 or not x_dev.is_cuda or not x_dev.is_contiguous():
+        raise ValueError("x must be a contiguous CUDA bfloat16 tensor")
+    C = x_dev.shape[-1]
+    rows = x_dev.numel() // C
+    out = torch.empty(rows, dtype=torch.uint8, device=x_dev.device)
+    _check(lib().asx_mask_from_activation(x_dev.data_ptr(), rows, C, out.data_ptr(), _stream_ptr(stream)),
+           "asx_mask_from_activation")
     return out
 
 

@@ -586,6 +586,18 @@ asx_status asx_compact(const uint8_t* mask_dev, int64_t rows, int32_t* kept_dev,
                                     static_cast<cudaStream_t>(cuda_stream)));
 }
 
+asx_status asx_mask_from_activation(const void* x_dev, int64_t rows, int C, uint8_t* mask_dev, void* cuda_stream)
+{
+    if (rows < 0 || rows >= (1ll << 31) || C < 1 || C > (1 << 20)) return ASX_ERR_INVALID_ARG;
+    if (rows > 0 && (x_dev == nullptr || mask_dev == nullptr)) return ASX_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(x_dev) & 1) return ASX_ERR_ALIGN;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        return ASX_ERR_CUDA;
+    return from_cuda(launch_mask_from_activation(x_dev, rows, C, mask_dev, sms, static_cast<cudaStream_t>(cuda_stream)));
+}
+
 asx_status asx_compact_status(const void* scratch_dev, void* cuda_stream)
 {
     if (scratch_dev == nullptr) return ASX_ERR_INVALID_ARG;
