@@ -399,11 +399,28 @@ def run_ours(args):
     h2d = sum(L.x_host.numel() * 2 for L in layers)
     d2h = sum(L.y_host.numel() * 2 for L in layers)
 
+    # Copies in, kernels and copies out run on three streams, ordered per layer by events, so that the
+    # two directions of the host link and the kernels overlap across layers and steps; every step still
+    # copies every layer's input from pinned host memory and every output back.
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in layers]
+    ev_done = [torch.cuda.Event() for _ in layers]
+    ev_out = [torch.cuda.Event() for _ in layers]
+
     def e2e_step():
-        for L in layers:
-            L.x.copy_(L.x_host, non_blocking=True)
+        for i, L in enumerate(layers):
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(ev_done[i])             # the previous step's kernel has read x
+                L.x.copy_(L.x_host, non_blocking=True)
+                ev_in[i].record(s_in)
+            st_obj.wait_event(ev_in[i])
+            st_obj.wait_event(ev_out[i])                # the previous step's copy of y has left
             L.step(st, RELU)
-            L.y_host.copy_(L.y, non_blocking=True)
+            ev_done[i].record(st_obj)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[i])
+                L.y_host.copy_(L.y, non_blocking=True)
+                ev_out[i].record(s_out)
     e2e_step()
     barrier()
     tw0 = time.perf_counter()
