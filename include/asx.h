@@ -53,7 +53,9 @@ typedef enum {
 enum {
     ASX_ACT_RELU = 1,      /* y = max(acc + bias, 0) on kept rows (default: acc + bias) */
     ASX_RECOMPACT = 2,     /* rebuild the kept-row list from the stored mask inside this call */
-    ASX_IMPL_NAIVE = 4     /* run the slow one-thread-per-output CUDA kernel (debug reference) */
+    ASX_IMPL_NAIVE = 4,    /* run the slow one-thread-per-output CUDA kernel (debug reference) */
+    ASX_OUT_COMPACT = 8,   /* y holds the kept rows only: [Nb*P'][C_out] in kept order, nothing zero-filled */
+    ASX_IN_COMPACT = 16    /* x holds only the positions kept by the mask given to asx_set_input_mask */
 };
 
 /* Human-readable name of a status code; never NULL; static storage. */
@@ -115,6 +117,23 @@ asx_status asx_set_mask_from_scores(asx_layer* layer, const float* score, int H0
                                     double sparsity, void* cuda_stream);
 
 /*
+ * Layer chaining without re-densifying.  The paper expands every masked layer's output back to the
+ * dense shape only because "the subsequent layer assumes dense activation" (Section 3.2, stage
+ * iii) and names that post-processing as one of its two overheads (Section 4.3).  Here a layer run
+ * with ASX_OUT_COMPACT writes row j of the kept list of image n at y[n*P' + j][0..C_out) and writes
+ * nothing else, and the layer that consumes it is run with ASX_IN_COMPACT after being told the
+ * producer's mask with asx_set_input_mask: its gather then reads input position p of image n at
+ * x[n*P'_in + rank(p)] when p was kept and zeros when it was dropped, which is what the dense
+ * tensor would have held.
+ *   mask : `rows` bytes (0 / non-zero), host or device pointer (a device mask is copied to the host,
+ *          which waits for it); rows must equal H*W of the tensors this layer is run on (one mask
+ *          per image, shared by the batch).  0 < rows < 2^31.
+ * ASX_IN_COMPACT needs C_in % 8 == 0 and at least one kept input position (else ASX_ERR_UNSUPPORTED),
+ * and is not available with ASX_IMPL_NAIVE.
+ */
+asx_status asx_set_input_mask(asx_layer* layer, const uint8_t* mask, int64_t rows, void* cuda_stream);
+
+/*
  * Rebuild the kept-row list from the stored mask (stage i alone; the same work the
  * ASX_RECOMPACT flag does inside asx_run).  Asynchronous on `cuda_stream`; allocates nothing.
  * ASX_ERR_NO_MASK before any asx_set_mask*.
@@ -130,7 +149,9 @@ asx_status asx_recompact(asx_layer* layer, void* cuda_stream);
  *   bias : device, fp32 [C_out], 4-byte aligned, or NULL for zero bias.
  *   y    : device, bf16 [Nb][Ho][Wo][C_out], Ho = (H + 2*pad - kh)/stride + 1 (Wo alike);
  *          16-byte aligned when C_out % 8 == 0, else 2-byte; must not overlap x.
- *   flags: OR of ASX_ACT_RELU, ASX_RECOMPACT, ASX_IMPL_NAIVE.
+ *   flags: OR of ASX_ACT_RELU, ASX_RECOMPACT, ASX_IMPL_NAIVE, ASX_OUT_COMPACT, ASX_IN_COMPACT.  With
+ *          ASX_OUT_COMPACT y is bf16 [Nb*P'][C_out] (P' = kept entries of the mask, which must then be
+ *          shared by the batch); with ASX_IN_COMPACT x is bf16 [Nb*P'_in][C_in] (see asx_set_input_mask).
  * Asynchronous on `cuda_stream`.  Allocates in two cases only, on first use and when the buffers
  * must grow: when C_in % 8 != 0 the layer keeps copies of x and w with the channels zero-padded to
  * a multiple of 8 (refreshed by a small kernel on every call); and when a layer has far fewer

@@ -9,14 +9,14 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libasx.so")
 _lib = None
 
-ACT_RELU, RECOMPACT, IMPL_NAIVE = 1, 2, 4
+ACT_RELU, RECOMPACT, IMPL_NAIVE, OUT_COMPACT, IN_COMPACT = 1, 2, 4, 8, 16
 
 # every symbol include/asx.h declares
 EXPORTS = (
     "asx_status_string", "asx_create_layer", "asx_set_mask", "asx_set_mask_random", "asx_recompact", "asx_run",
     "asx_get_kept", "asx_get_kept_host", "asx_get_mask", "asx_last_device_status", "asx_destroy",
     "asx_compact_scratch_bytes", "asx_compact", "asx_compact_status", "asx_compact_static",
-    "asx_mask_from_scores", "asx_set_mask_from_scores", "asx_mask_from_activation",
+    "asx_mask_from_scores", "asx_set_mask_from_scores", "asx_mask_from_activation", "asx_set_input_mask",
 )
 COMPACT_STATIC_MAX_ROWS = 1 << 24
 
@@ -58,6 +58,7 @@ def lib():
         L.asx_compact.argtypes = [vp, i64, vp, vp, vp, i64, vp]
         L.asx_compact_status.argtypes = [vp, vp]
         L.asx_compact_static.argtypes = [vp, i64, vp, vp, vp]
+        L.asx_set_input_mask.argtypes = [vp, vp, i64, vp]
         L.asx_mask_from_activation.argtypes = [vp, i64, ci, vp, vp]
         L.asx_mask_from_scores.argtypes = [vp, ci, ci, ci, ci, ctypes.c_double, vp]
         L.asx_set_mask_from_scores.argtypes = [vp, vp, ci, ci, ci, ci, ctypes.c_double, vp]
@@ -105,6 +106,20 @@ class MaskedConvLayer:
             m = np.ascontiguousarray(mask, dtype=np.uint8)
             ptr, rows = m.ctypes.data, m.size
         _check(lib().asx_set_mask(self._h, ptr, rows, _stream_ptr(stream)), "asx_set_mask")
+
+    def set_input_mask(self, mask, stream=None) -> None:
+        """The mask of the layer that produced this layer's (compact) input; see ASX_IN_COMPACT."""
+        import numpy as np
+        import torch
+        if isinstance(mask, torch.Tensor):
+            m = mask.contiguous()
+            if m.dtype != torch.uint8:
+                raise TypeError("mask must be uint8")
+            ptr, rows = m.data_ptr(), m.numel()
+        else:
+            m = np.ascontiguousarray(mask, dtype=np.uint8)
+            ptr, rows = m.ctypes.data, m.size
+        _check(lib().asx_set_input_mask(self._h, ptr, rows, _stream_ptr(stream)), "asx_set_input_mask")
 
     def set_mask_random(self, rows: int, sparsity: float, block: int, seed: int, stream=None) -> None:
         _check(lib().asx_set_mask_random(self._h, rows, float(sparsity), block, seed, _stream_ptr(stream)),

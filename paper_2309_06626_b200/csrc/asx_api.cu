@@ -24,6 +24,9 @@ struct asx_layer {
     int32_t* d_small = nullptr;        // [0] kept count, [1] status word
     bool has_mask = false;
     int64_t host_kept = -1;            // kept entries of the mask when it came from the host, else -1
+    int32_t* d_in_rank = nullptr;      // compact input: row of each input position within its image, -1 = dropped
+    int64_t in_rows = 0, in_rank_cap = 0;
+    int64_t in_kept = 0;
     // staging copies with zero-padded channels, for C_in not a multiple of 8
     void* d_wpack = nullptr;
     size_t wpack_bytes = 0;
@@ -278,6 +281,49 @@ asx_status asx_set_mask_from_scores(asx_layer* L, const float* score, int H0, in
     return asx_set_mask(L, mask.data(), (int64_t)Ho * Wo, cuda_stream);
 }
 
+asx_status asx_set_input_mask(asx_layer* L, const uint8_t* mask, int64_t rows, void* cuda_stream)
+{
+    if (L == nullptr || mask == nullptr || rows < 1 || rows >= (1ll << 31)) return ASX_ERR_INVALID_ARG;
+    const asx_status s = bind_device(L);
+    if (s != ASX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    std::vector<uint8_t> host;
+    std::vector<int32_t> rank;
+    try {
+        host.resize((size_t)rows);
+        rank.resize((size_t)rows);
+    } catch (const std::bad_alloc&) {
+        return ASX_ERR_OOM;
+    }
+    cudaPointerAttributes attr;
+    const bool on_device = cudaPointerGetAttributes(&attr, mask) == cudaSuccess &&
+                           (attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged);
+    if (on_device) {
+        if (cudaStreamSynchronize(st) != cudaSuccess) return ASX_ERR_CUDA;        // whatever writes the mask is on this stream
+        if (cudaMemcpy(host.data(), mask, (size_t)rows, cudaMemcpyDeviceToHost) != cudaSuccess) return ASX_ERR_CUDA;
+    } else {
+        cudaGetLastError();
+        std::memcpy(host.data(), mask, (size_t)rows);
+    }
+    int32_t kept = 0;
+    for (int64_t p = 0; p < rows; ++p) rank[(size_t)p] = host[(size_t)p] != 0 ? kept++ : -1;
+    if (rows > L->in_rank_cap) {
+        if (cudaStreamSynchronize(L->last_stream) != cudaSuccess) return ASX_ERR_CUDA;
+        cudaFree(L->d_in_rank);
+        L->d_in_rank = nullptr; L->in_rank_cap = 0;
+        if (cudaMalloc(&L->d_in_rank, (size_t)rows * sizeof(int32_t)) != cudaSuccess) return ASX_ERR_OOM;
+        L->in_rank_cap = rows;
+    }
+    // a launch that still reads the old table is ordered before this copy when it used the same stream
+    if (cudaMemcpyAsync(L->d_in_rank, rank.data(), (size_t)rows * sizeof(int32_t), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return ASX_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ASX_ERR_CUDA;            // `rank` goes out of scope
+    L->in_rows = rows;
+    L->in_kept = kept;
+    L->last_stream = st;
+    return ASX_OK;
+}
+
 asx_status asx_recompact(asx_layer* L, void* cuda_stream)
 {
     if (L == nullptr) return ASX_ERR_INVALID_ARG;
@@ -293,7 +339,8 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
 {
     if (L == nullptr || x == nullptr || w == nullptr || y == nullptr) return ASX_ERR_INVALID_ARG;
     if (Nb < 1 || H < 1 || W < 1) return ASX_ERR_INVALID_ARG;
-    if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE)) return ASX_ERR_INVALID_ARG;
+    if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE | ASX_OUT_COMPACT | ASX_IN_COMPACT)) return ASX_ERR_INVALID_ARG;
+    if ((flags & ASX_IMPL_NAIVE) && (flags & (ASX_OUT_COMPACT | ASX_IN_COMPACT))) return ASX_ERR_INVALID_ARG;
     if (H + 2 * L->pad < L->kh || W + 2 * L->pad < L->kw) return ASX_ERR_INVALID_ARG;
     if (!L->has_mask) return ASX_ERR_NO_MASK;
     asx_status s = bind_device(L);
@@ -312,6 +359,14 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     if (M > lim || (int64_t)Nb * H * W * L->C_in > lim || M * L->C_out > lim) return ASX_ERR_UNSUPPORTED;
     if (L->rows != P && L->rows != M) return ASX_ERR_SHAPE;
     g.P = (int)P; g.M = (int)M; g.rows = (int)L->rows;
+    const bool in_compact = (flags & ASX_IN_COMPACT) != 0, out_compact = (flags & ASX_OUT_COMPACT) != 0;
+    if (out_compact && L->rows != P) return ASX_ERR_SHAPE;            // kept order n*P' + j needs one mask for the batch
+    if (in_compact) {
+        if (L->d_in_rank == nullptr) return ASX_ERR_NO_MASK;
+        if (L->in_rows != (int64_t)H * W) return ASX_ERR_SHAPE;
+        if (L->C_in % 8 != 0 || L->in_kept < 1) return ASX_ERR_UNSUPPORTED;
+    }
+    const int64_t x_rows = in_compact ? (int64_t)Nb * L->in_kept : (int64_t)Nb * H * W;     // rows of x in memory
 
     const bool vec_in = (L->C_in % 8 == 0);
     const uintptr_t in_align = vec_in ? 15 : 1;
@@ -320,7 +375,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     if (reinterpret_cast<uintptr_t>(y) & ((L->C_out % 8 == 0) ? 15 : 1)) return ASX_ERR_ALIGN;
     if (bias != nullptr && (reinterpret_cast<uintptr_t>(bias) & 3)) return ASX_ERR_ALIGN;
     {
-        const uintptr_t xb = reinterpret_cast<uintptr_t>(x), xe = xb + (uintptr_t)Nb * H * W * L->C_in * 2;
+        const uintptr_t xb = reinterpret_cast<uintptr_t>(x), xe = xb + (uintptr_t)x_rows * L->C_in * 2;
         const uintptr_t yb = reinterpret_cast<uintptr_t>(y), ye = yb + (uintptr_t)M * L->C_out * 2;
         if (xb < ye && yb < xe) return ASX_ERR_INVALID_ARG;
     }
@@ -358,7 +413,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     // a view whose rows are 32 bytes apart (rows overlap; the borders make every tap in bounds).
     // shift = pad & 1 aligns the window to the blocks; the filter gets zero rows / columns there.
     const int bshift = L->pad & 1;
-    const bool blocks2x2 = L->C_in <= 4 && L->stride == 2 && (W % 2) == 0 && (H % 2) == 0 &&
+    const bool blocks2x2 = !in_compact && L->C_in <= 4 && L->stride == 2 && (W % 2) == 0 && (H % 2) == 0 &&
                            (L->kw + bshift + 1) / 2 == 4 && L->kh + bshift <= 32;
     if (blocks2x2) {
         const int kh2 = (L->kh + bshift + 1) / 2;
@@ -484,7 +539,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         L->tmap_ptr = wsrc; L->tmap_BN = plan.BN; L->tmap_Kw = Kw;
     }
     if (plan.vec == 2) {
-        const int64_t pixels = (int64_t)Nb * g.H * g.W;
+        const int64_t pixels = in_compact ? x_rows : (int64_t)Nb * g.H * g.W;
         const int row_stride = x_row_stride ? x_row_stride : g.C_in * 2;
         if (L->tmapx_ptr != xsrc || L->tmapx_pixels != pixels || L->tmapx_stride != row_stride) {
             EncodeTiledFn enc = encode_tiled_fn();
@@ -501,7 +556,8 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         }
     }
     return from_cuda(launch_fast(g, plan, L->tmap, plan.vec == 2 ? L->tmap_x : L->tmap, xsrc, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
-                                 L->num_sms, fuse_compact ? 1 : 0, L->host_kept, static_cast<float*>(L->d_ws), L->d_wscnt, st));
+                                 L->num_sms, fuse_compact ? 1 : 0, L->host_kept, static_cast<float*>(L->d_ws), L->d_wscnt,
+                                 out_compact ? 1 : 0, in_compact ? L->d_in_rank : nullptr, (int)L->in_kept, st));
 }
 
 asx_status asx_get_kept(asx_layer* L, int64_t* count, const int32_t** dev_kept)
@@ -562,7 +618,7 @@ asx_status asx_destroy(asx_layer* L)
     if (L->device >= 0) {
         cudaStreamSynchronize(L->last_stream);
         cudaFree(L->d_mask); cudaFree(L->d_kept); cudaFree(L->d_scratch);
-        cudaFree(L->d_small); cudaFree(L->d_wpack); cudaFree(L->d_xpad); cudaFree(L->d_ws); cudaFree(L->d_wscnt);
+        cudaFree(L->d_small); cudaFree(L->d_wpack); cudaFree(L->d_xpad); cudaFree(L->d_ws); cudaFree(L->d_wscnt); cudaFree(L->d_in_rank);
     }
     delete L;
     return ASX_OK;

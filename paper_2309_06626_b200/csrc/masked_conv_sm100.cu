@@ -92,6 +92,10 @@ struct FastArgs {
     int fuse_compact;   // rebuild the kept-row list from the mask inside this kernel (small masks)
     int32_t* kept_out;  // where the fused compaction writes the list and its count
     int32_t* count_out;
+    int out_compact;    // y holds the kept rows only, in kept order (row rk at y[rk][*]); nothing is zero-filled
+    const int32_t* in_rank;   // non-null: x holds only the rows its own mask kept; in_rank[pos] = row of input position
+                              // pos within its image's in_kept rows, or -1 for a dropped position (read as zeros)
+    int in_kept;        // kept input positions per image
     int ksplit;         // work items per output tile: each takes a contiguous share of the k-blocks
     float* ws_partial;  // ksplit > 1: [item][128][BN] fp32 partial tiles
     int* ws_counters;   // ksplit > 1: per output tile {partials written, slices reduced}, zero between launches
@@ -271,7 +275,8 @@ __device__ __forceinline__ Item item_of(int t, int KB, const FastArgs& a)
 }
 
 // What the gather warps need to know about the rk-th kept lowered row: the pixel index of its
-// window's corner, (n H + iy0) W + ix0, and the corner's coordinates packed as iy0 << 16 | ix0.
+// window's corner, (n H + iy0) W + ix0 (with a compact input: the first input row of its image,
+// n * in_kept), and the corner's coordinates packed as iy0 << 16 | ix0.
 // Rows past the end get iy0 = -32768, for which no filter tap is inside the image.
 __device__ __forceinline__ int2 row_info_of(int rk, int Mk, const FastDiv& fdcnt, const ConvGeom& g, const FastArgs& a,
                                             const KeptList& kept)
@@ -283,7 +288,7 @@ __device__ __forceinline__ int2 row_info_of(int rk, int Mk, const FastDiv& fdcnt
             const int n = (int)fd_div((uint32_t)row, a.fdP), p = row - n * g.P;
             const int oy = (int)fd_div((uint32_t)p, a.fdWo), ox = p - oy * g.Wo;
             const int iy0 = oy * g.stride - g.pad, ix0 = ox * g.stride_w - g.pad_w;
-            info.x = (n * g.H + iy0) * g.W + ix0;
+            info.x = a.in_rank != nullptr ? n * a.in_kept : (n * g.H + iy0) * g.W + ix0;
             info.y = (iy0 << 16) | (ix0 & 0xffff);
         } else {
             atomicOr(a.dev_status, DEV_BAD_INDEX);
@@ -292,7 +297,7 @@ __device__ __forceinline__ int2 row_info_of(int rk, int Mk, const FastDiv& fdcnt
     return info;
 }
 
-template <int MODE>
+template <int MODE, bool IN_COMPACT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                          const ConvGeom g, const FastArgs a)
@@ -496,7 +501,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             const uint32_t use = (uint32_t)(ti >> 1) & 1u;
             const int rk = m_tile * BM + q * 32 + lane;
             const bool valid = rk < Mk;
-            const long long yoff = valid ? (long long)out_row_of(rk, fdcnt, g, kept_list) * N : 0;
+            const long long yoff = valid ? (long long)(a.out_compact ? rk : out_row_of(rk, fdcnt, g, kept_list)) * N : 0;
             {
                 float* sb = sh->bias[buf];
                 const int et = (warp - WARP_EPI0) * 32 + lane;
@@ -563,7 +568,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                 const float4* __restrict__ tile_ws = reinterpret_cast<const float4*>(a.ws_partial) + (size_t)item.tile * a.ksplit * (BN >> 2) * BM;
                 uint4* __restrict__ yv = reinterpret_cast<uint4*>(a.y);
                 const int rk2 = m_tile * BM + et;              // NUM_EPI_WARPS * 32 == BM: thread et owns row et
-                const long long yrow = rk2 < Mk ? (long long)out_row_of(rk2, fdcnt, g, kept_list) * N : -1;
+                const long long yrow = rk2 < Mk ? (long long)(a.out_compact ? rk2 : out_row_of(rk2, fdcnt, g, kept_list)) * N : -1;
 #pragma unroll 2
                 for (int gq = g_lo; gq < g_hi; ++gq) {
                     if (yrow < 0 || n0 + gq * 8 >= N) continue;
@@ -656,6 +661,8 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[buf]));
         }
+    } else if (warp >= WARP_ZERO0 && a.out_compact) {
+        // a compact output has no dropped rows
     } else if (warp >= WARP_ZERO0) {   // (the row-coordinate warp was handled above)
         // ------------------------------------------------------------------ zeros for dropped rows
         // Algorithm 2's post-processing writes zeros wherever the mask is 0.  These warps stream
@@ -729,7 +736,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             // the stage's barrier by the filter thread.  A row gather costs its warp about 100
             // cycles plus 56 per further lane, hence few issuing lanes in many warps.
             if (lane < 4) {
-                const int oob = g.Nb * g.H * g.W;
+                const int oob = IN_COMPACT ? g.Nb * a.in_kept : g.Nb * g.H * g.W;
                 int s = 0, j = 0, it = 0;
                 uint32_t ph = 0;
                 bool ok = true;
@@ -757,7 +764,13 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
                                 const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
-                                idx[i] = ((unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W) ? pix[i] + koff : oob;
+                                const bool in = (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
+                                if (!IN_COMPACT) {
+                                    idx[i] = in ? pix[i] + koff : oob;
+                                } else {               // compact input: a dropped position reads zeros like padding
+                                    const int rnk = in ? __ldg(a.in_rank + iy * g.W + ix) : -1;
+                                    idx[i] = rnk >= 0 ? pix[i] + rnk : oob;
+                                }
                             }
                             if (!wait_bar<20>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
                             ptx::tma_gather4_2d(smem_base + s * stage_bytes + (uint32_t)(16 * pwg + 4 * lane) * 128u, &tmap_x,
@@ -821,9 +834,15 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
-                        const bool in = kvalid && (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
+                        bool in = kvalid && (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
+                        int off = base[i] + tapoff;
+                        if (IN_COMPACT) {                      // compact input: base is the image's first row
+                            const int rnk = in ? __ldg(a.in_rank + iy * g.W + ix) : -1;
+                            in = rnk >= 0;
+                            off = base[i] + rnk * g.C_in + ci;
+                        }
                         ptx::cp_async_16(stage + ((i & 1) ? dst_b : dst_a) + (uint32_t)((i >> 1) * 1024),
-                                         x2 + (in ? base[i] + tapoff : 0), in ? 16u : 0u);
+                                         x2 + (in ? off : 0), in ? 16u : 0u);
                     }
                     ptx::cp_async_mbar_arrive_noinc(ptx::smem_u32(&sh->full[s]));
                     tap += adv_tap;
@@ -1024,7 +1043,7 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
                         const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
                         int num_sms, int fuse_compact, long long host_kept, float* ws_partial, int* ws_counters,
-                        cudaStream_t st)
+                        int out_compact, const int32_t* in_rank, int in_kept, cudaStream_t st)
 {
     FastArgs a;
     a.fdcnt_host = make_fastdiv((uint32_t)(host_kept > 0 && host_kept < (1ll << 31) ? host_kept : 1));
@@ -1040,6 +1059,9 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     a.count = count;
     a.dev_status = dev_status;
     a.relu = relu;
+    a.out_compact = out_compact;
+    a.in_rank = in_rank;
+    a.in_kept = in_kept;
     a.BN = plan.BN;
     a.fdP = make_fastdiv((uint32_t)g.P);
     a.fdWo = make_fastdiv((uint32_t)g.Wo);
@@ -1062,12 +1084,16 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     long long tiles = ((long long)g.M + BM - 1) / BM * plan.n_tiles * plan.ksplit;
     int grid = (int)(tiles < num_sms ? tiles : num_sms);
     if (grid < 1) grid = 1;
-    auto kern = plan.vec == GATHER_TMA ? masked_conv_sm100_kernel<GATHER_TMA> : masked_conv_sm100_kernel<GATHER_CPASYNC>;
-    static int smem_set[3] = {0, 0, 0};         // largest dynamic shared memory size enabled so far
-    if (plan.smem_bytes > smem_set[plan.vec]) {
+    const int variant = plan.vec + (in_rank != nullptr ? 2 : 0);      // 1, 2: dense input; 3, 4: compact input
+    auto kern = variant == 2   ? masked_conv_sm100_kernel<GATHER_TMA, false>
+                : variant == 1 ? masked_conv_sm100_kernel<GATHER_CPASYNC, false>
+                : variant == 4 ? masked_conv_sm100_kernel<GATHER_TMA, true>
+                               : masked_conv_sm100_kernel<GATHER_CPASYNC, true>;
+    static int smem_set[5] = {0, 0, 0, 0, 0};   // largest dynamic shared memory size enabled so far, per variant
+    if (plan.smem_bytes > smem_set[variant]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
         if (e != cudaSuccess) return e;
-        smem_set[plan.vec] = plan.smem_bytes;
+        smem_set[variant] = plan.smem_bytes;
     }
     return launch_pdl(kern, dim3(grid), dim3(NUM_THREADS), (size_t)plan.smem_bytes, st, tmap_w, tmap_x, g, a);
 }

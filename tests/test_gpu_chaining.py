@@ -1,0 +1,102 @@
+"""Layer chaining without re-densifying (compact outputs and inputs) against the oracle.
+
+The oracle has no notion of compact tensors: a compact output must equal the kept rows of the
+oracle's dense output, and a convolution fed with a compact input must equal the oracle's
+convolution of the dense tensor that has zeros at the dropped positions."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2309_06626_b200 as asx
+import workloads as wl
+from gpu_util import to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_raw(layer, x_dev, Nb, H, W, w_dev, b_dev, y_dev, flags):
+    st = int(torch.cuda.current_stream().cuda_stream)
+    rc = layer.run_raw(x_dev.data_ptr(), Nb, H, W, w_dev.data_ptr(), b_dev.data_ptr() if b_dev is not None else 0,
+                       y_dev.data_ptr(), flags, st)
+    assert rc == 0, f"asx_run returned {rc}"
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0
+
+
+def _rel(a, b):
+    return np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30)
+
+
+CASES = [
+    # C_in, C_mid, C_out, k1, s1, p1, k2, s2, p2, H, W, Nb, sparsity1 %, sparsity2 %, block
+    (64, 64, 48, 3, 1, 1, 3, 1, 1, 20, 23, 2, 40, 30, 1),        # TMA gather on both layers
+    (16, 32, 24, 3, 2, 1, 3, 1, 1, 29, 31, 2, 50, 50, 4),        # cp.async gather on the second layer
+    (64, 128, 256, 1, 1, 0, 3, 2, 1, 14, 14, 3, 25, 60, 2),      # 1x1 then a strided 3x3
+    (128, 512, 64, 3, 1, 1, 3, 1, 1, 7, 7, 4, 50, 50, 1),        # few rows, long reduction: shared k-blocks on layer 2
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=[f"c{i}" for i in range(len(CASES))])
+def test_two_layers_chained_compact(case):
+    cin, cmid, cout, k1, s1, p1, k2, s2, p2, H, W, Nb, sp1, sp2, blk = case
+    l1 = wl.LayerSpec("chain1", cin, cmid, k1, k1, s1, p1, H, W, Nb, sp1, blk, "relu", wl.BASE_SEED + 301)
+    l2 = wl.LayerSpec("chain2", cmid, cout, k2, k2, s2, p2, l1.Ho, l1.Wo, Nb, sp2, blk, "relu", wl.BASE_SEED + 302)
+    x, w1, b1, m1 = wl.make_x(l1), wl.make_w(l1), wl.make_b(l1), wl.make_layer_mask(l1)
+    w2, b2, m2 = wl.make_w(l2), wl.make_b(l2), wl.make_layer_mask(l2)
+    # oracle: two dense layers; the intermediate is stored as bf16 by the GPU path
+    y1_ref = oracle.masked_conv(x, w1, b1, m1, s1, p1, True)
+    y1_bf = oracle.bf16_round(y1_ref.astype(np.float32)).astype(np.float64)
+    y2_ref = oracle.masked_conv(y1_bf.astype(np.float32), w2, b2, m2, s2, p2, True)
+
+    kept1, kept2 = int(m1.sum()), int(m2.sum())
+    A = asx.MaskedConvLayer(cin, cmid, k1, k1, s1, p1)
+    B = asx.MaskedConvLayer(cmid, cout, k2, k2, s2, p2)
+    A.set_mask(m1)
+    B.set_mask(m2)
+    B.set_input_mask(m1)
+    xd, w1d, w2d = to_dev_bf16(x), to_dev_bf16(w1), to_dev_bf16(w2)
+    b1d, b2d = torch.from_numpy(b1).cuda(), torch.from_numpy(b2).cuda()
+    y1c = torch.full((Nb * kept1, cmid), float("nan"), dtype=torch.bfloat16, device="cuda")
+    y2c = torch.full((Nb * kept2, cout), float("nan"), dtype=torch.bfloat16, device="cuda")
+    _run_raw(A, xd, Nb, H, W, w1d, b1d, y1c, asx.ACT_RELU | asx.RECOMPACT | asx.OUT_COMPACT)
+    _run_raw(B, y1c, Nb, l1.Ho, l1.Wo, w2d, b2d, y2c, asx.ACT_RELU | asx.RECOMPACT | asx.IN_COMPACT | asx.OUT_COMPACT)
+    A.close(); B.close()
+
+    rows1 = (np.arange(Nb)[:, None] * l1.P + np.flatnonzero(m1)[None, :]).reshape(-1)
+    rows2 = (np.arange(Nb)[:, None] * l2.P + np.flatnonzero(m2)[None, :]).reshape(-1)
+    got1 = y1c.float().cpu().numpy().astype(np.float64)
+    got2 = y2c.float().cpu().numpy().astype(np.float64)
+    assert not np.isnan(got1).any() and not np.isnan(got2).any(), "a compact row was never written"
+    assert _rel(got1, y1_ref.reshape(l1.M, cmid)[rows1]) < 5e-3
+    assert _rel(got2, y2_ref.reshape(l2.M, cout)[rows2]) < 5e-3
+
+
+def test_compact_input_into_dense_output_and_errors():
+    spec = wl.LayerSpec("cin_only", 64, 64, 3, 3, 1, 1, 17, 19, 2, 30, 1, "relu", wl.BASE_SEED + 303)
+    x, w, b, m = wl.make_x(spec), wl.make_w(spec), wl.make_b(spec), wl.make_layer_mask(spec)
+    rng = np.random.default_rng(4)
+    m_in = (rng.random(spec.H * spec.W) < 0.6).astype(np.uint8)
+    x_masked = x * np.tile(m_in, spec.Nb).reshape(spec.Nb, spec.H, spec.W, 1)
+    ref = oracle.masked_conv(x_masked, w, b, m, spec.stride, spec.pad, True)
+    rows_in = (np.arange(spec.Nb)[:, None] * spec.H * spec.W + np.flatnonzero(m_in)[None, :]).reshape(-1)
+    xc = to_dev_bf16(x.reshape(-1, spec.C_in)[rows_in])
+    layer = asx.MaskedConvLayer(spec.C_in, spec.C_out, 3, 3, 1, 1)
+    layer.set_mask(m)
+    wd, bd = to_dev_bf16(w), torch.from_numpy(b).cuda()
+    y = torch.full((spec.Nb, spec.Ho, spec.Wo, spec.C_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+    st = int(torch.cuda.current_stream().cuda_stream)
+    args = (xc.data_ptr(), spec.Nb, spec.H, spec.W, wd.data_ptr(), bd.data_ptr(), y.data_ptr())
+    assert layer.run_raw(*args, asx.ACT_RELU | asx.IN_COMPACT, st) == 3                       # no input mask yet
+    layer.set_input_mask(torch.from_numpy(m_in).cuda())                                       # from device memory
+    assert layer.run_raw(*args, asx.ACT_RELU | asx.IN_COMPACT | asx.IMPL_NAIVE, st) == 1      # not with the reference kernel
+    assert layer.run_raw(xc.data_ptr(), spec.Nb, spec.H + 1, spec.W, wd.data_ptr(), bd.data_ptr(), y.data_ptr(),
+                         asx.ACT_RELU | asx.IN_COMPACT, st) in (4,)                            # mask length != H*W
+    assert layer.run_raw(*args, asx.ACT_RELU | asx.IN_COMPACT, st) == 0
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0
+    layer.close()
+    got = y.float().cpu().numpy().astype(np.float64).reshape(ref.shape)
+    assert not np.isnan(got).any()
+    assert _rel(got, ref) < 5e-3
+    assert not got.reshape(spec.M, -1)[np.tile(m, spec.Nb) == 0].any()
