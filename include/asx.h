@@ -40,7 +40,7 @@ typedef struct asx_layer asx_layer;   /* opaque, owned by the library */
 typedef enum {
     ASX_OK = 0,
     ASX_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, unknown flag */
-    ASX_ERR_UNSUPPORTED = 2,   /* a legal convolution this build cannot run */
+    ASX_ERR_UNSUPPORTED = 2,   /* a legal convolution this library cannot run */
     ASX_ERR_NO_MASK = 3,       /* asx_run before any asx_set_mask* */
     ASX_ERR_SHAPE = 4,         /* mask length does not match the output geometry */
     ASX_ERR_ALIGN = 5,         /* a pointer is not aligned as documented */
