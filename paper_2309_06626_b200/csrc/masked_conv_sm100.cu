@@ -634,7 +634,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
 #pragma unroll
                     for (int h = 0; h < 4; ++h) {
                         const int colh = col0 + 8 * h;
-                        if (colh >= N) break;
+                        if (colh >= N || c0 + 8 * h >= BN) break;      // the tile's last chunk may be 16 columns wide
                         float v[8];
 #pragma unroll
                         for (int j = 0; j < 8; ++j) {

@@ -1,0 +1,42 @@
+"""Seeded random layer geometries against the oracle: channel counts around every staging path
+(1..6, multiples of 8 and 64, odd counts), filter sizes 1..8, strides 1..3, paddings up to the
+filter size, ragged images, shared and per-row masks, with and without bias and ReLU."""
+import numpy as np
+import pytest
+
+import paper_2309_06626_b200 as asx
+import workloads as wl
+from gpu_util import check_against_oracle, make_problem
+
+pytestmark = pytest.mark.gpu
+
+
+def _random_spec(i):
+    rng = np.random.default_rng(90_000 + i)
+    cin = int(rng.choice([1, 2, 3, 4, 5, 6, 8, 16, 24, 32, 40, 64, 64, 96, 128, 192, 256]))
+    cout = int(rng.choice([1, 7, 8, 16, 24, 40, 64, 64, 72, 128, 136, 256, 264]))
+    k = int(rng.choice([1, 2, 3, 3, 3, 4, 5, 7, 8]))
+    stride = int(rng.choice([1, 1, 2, 2, 3]))
+    pad = int(rng.integers(0, k))                      # 0 .. k-1
+    # keep K = k*k*cin moderate so that the oracle stays fast
+    while k * k * cin > 6000:
+        cin //= 2
+    H = int(rng.integers(max(k - 2 * pad, 1) + 2, 34))
+    W = int(rng.integers(max(k - 2 * pad, 1) + 2, 34))
+    if rng.random() < 0.5:                             # even sizes reach the pixel-pair and 2x2-block forms
+        H += H % 2
+        W += W % 2
+    Nb = int(rng.integers(1, 4))
+    pct = int(rng.choice([0, 10, 30, 50, 50, 75, 95, 100]))
+    block = int(rng.choice([1, 1, 2, 4, 16]))
+    return wl.LayerSpec(f"rnd{i}", cin, cout, k, k, stride, pad, H, W, Nb, pct, block, "relu", wl.BASE_SEED + 40_000 + i)
+
+
+@pytest.mark.parametrize("i", range(60))
+def test_random_geometry(i):
+    spec = _random_spec(i)
+    rng = np.random.default_rng(7 * i + 1)
+    per_row = bool(rng.random() < 0.3)
+    x, w, b, mask = make_problem(spec, per_row=per_row)
+    flags = (asx.ACT_RELU if rng.random() < 0.7 else 0) | (asx.RECOMPACT if rng.random() < 0.5 else 0)
+    check_against_oracle(spec, x, w, b if rng.random() < 0.8 else None, mask, flags)
