@@ -37,12 +37,12 @@ L2_BYTES = 126 * 1024 * 1024
 
 # DRAM traffic of the dominant kernel from one ncu capture of the default workload (ResNet-18 stack,
 # batch 64): dram__bytes_read.sum + dram__bytes_write.sum averaged over the 20 fused-kernel launches
-# of a step (12.17 MB read + 2.36 MB written; ncu flushes the caches before every captured launch,
+# of a step (12.17 MB read + 2.35 MB written; ncu flushes the caches before every captured launch,
 # so reads are cold-cache and most of a launch's output is still in L2 when its counters stop).
 # The figure belongs to the kernel sources whose digest is recorded with it; with any other sources
 # the bench reports null.
-NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.54e6,
-               "csrc_sha256": "05234a4221223ca1182c971895c6f8120c5e7f45c0facc9ff61f0f6ec641eca0"}
+NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.52e6,
+               "csrc_sha256": "5b9ab996dfb6ec012abca5f893de737b67910429bfbec173c2a6719cab59ca42"}
 
 
 def csrc_digest() -> str:
