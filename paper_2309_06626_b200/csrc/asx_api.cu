@@ -376,7 +376,9 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     if (bias != nullptr && (reinterpret_cast<uintptr_t>(bias) & 3)) return ASX_ERR_ALIGN;
     {
         const uintptr_t xb = reinterpret_cast<uintptr_t>(x), xe = xb + (uintptr_t)x_rows * L->C_in * 2;
-        const uintptr_t yb = reinterpret_cast<uintptr_t>(y), ye = yb + (uintptr_t)M * L->C_out * 2;
+        // a compact output holds Nb * P' rows (P' is known on the host for a mask that came from the host)
+        const int64_t y_rows = (out_compact && L->host_kept >= 0) ? (int64_t)Nb * L->host_kept : M;
+        const uintptr_t yb = reinterpret_cast<uintptr_t>(y), ye = yb + (uintptr_t)y_rows * L->C_out * 2;
         if (xb < ye && yb < xe) return ASX_ERR_INVALID_ARG;
     }
 

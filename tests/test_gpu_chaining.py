@@ -100,3 +100,22 @@ def test_compact_input_into_dense_output_and_errors():
     assert not np.isnan(got).any()
     assert _rel(got, ref) < 5e-3
     assert not got.reshape(spec.M, -1)[np.tile(m, spec.Nb) == 0].any()
+
+
+def test_compact_output_next_to_its_input_in_memory():
+    """A compact output is smaller than the dense one: an input that starts right behind it does not
+    overlap it (the overlap check once used the dense extent and refused such calls)."""
+    spec = wl.LayerSpec("adjacent", 8, 16, 3, 3, 1, 1, 12, 10, 1, 90, 1, "relu", wl.BASE_SEED + 304)
+    x, w, b, m = wl.make_x(spec), wl.make_w(spec), wl.make_b(spec), wl.make_layer_mask(spec)
+    kept = int(m.sum())
+    y_elems = ((kept * spec.C_out + 63) // 64) * 64                       # keeps x 16-byte aligned
+    arena = torch.zeros(y_elems + x.size, dtype=torch.bfloat16, device="cuda")
+    yc = arena[:kept * spec.C_out].view(kept, spec.C_out)
+    xd = arena[y_elems:].view(x.shape)
+    xd.copy_(to_dev_bf16(x))
+    layer = asx.MaskedConvLayer(spec.C_in, spec.C_out, 3, 3, 1, 1)
+    layer.set_mask(m)
+    _run_raw(layer, xd, 1, spec.H, spec.W, to_dev_bf16(w), torch.from_numpy(b).cuda(), yc, asx.ACT_RELU | asx.OUT_COMPACT)
+    layer.close()
+    ref = oracle.masked_conv(x, w, b, m, 1, 1, True).reshape(spec.M, spec.C_out)[np.flatnonzero(m)]
+    assert _rel(yc.float().cpu().numpy().astype(np.float64), ref) < 5e-3
