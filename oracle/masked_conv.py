@@ -15,6 +15,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "masked_conv_oracle.c")
+_SRC_ALG2 = os.path.join(_HERE, "alg2_fp32.c")      # the paper's three CPU stages in fp32 (a second baseline)
 _LIB = os.path.join(_HERE, "libasx_oracle.so")
 _lib = None
 
@@ -22,11 +23,11 @@ _lib = None
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc if the shared object is missing or stale."""
     if (not force and os.path.exists(_LIB)
-            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+            and os.path.getmtime(_LIB) >= max(os.path.getmtime(_SRC), os.path.getmtime(_SRC_ALG2))):
         return _LIB
     tmp = _LIB + f".tmp{os.getpid()}"
     subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-shared", "-fPIC",
-                           "-o", tmp, _SRC])
+                           "-o", tmp, _SRC, _SRC_ALG2])
     os.replace(tmp, _LIB)
     return _LIB
 
@@ -49,6 +50,8 @@ def _load():
         lib.asxo_masked_conv.restype = ci
         lib.asxo_masked_conv_rows.argtypes = conv_args + [i64p, i64, dp]
         lib.asxo_masked_conv_rows.restype = ci
+        lib.asxo_alg2_fp32.argtypes = [fp, ci, ci, ci, ci, fp, ci, ci, ci, ci, ci, fp, u8p, ci, fp]
+        lib.asxo_alg2_fp32.restype = ci
         _lib = lib
     return _lib
 
@@ -126,4 +129,27 @@ def masked_conv_rows(x, w, bias, mask, stride: int, pad: int, relu: bool, sel) -
         _ptr(sel, ctypes.c_int64), sel.size, _ptr(y, ctypes.c_double))
     if rc:
         raise ValueError(f"oracle rejected the arguments (code {rc})")
+    return y
+
+
+def alg2_fp32(x, w, bias: Optional[np.ndarray], mask, stride: int, pad: int, relu: bool) -> np.ndarray:
+    """Appendix A, Algorithm 2 as the paper runs it on a CPU, in fp32: indirection buffer over the
+    kept positions, dense product on the reduced range, reverse in-place expansion.  x [Nb][H][W][C_in],
+    w [C_out][kh][kw][C_in], mask of Ho*Wo entries (shared by the batch).  Returns fp32
+    [Nb][Ho][Wo][C_out].  Inputs are used as given (no bfloat16 rounding)."""
+    lib = _load()
+    x, w = _f32(x), _f32(w)
+    Nb, H, W, C_in = x.shape
+    C_out, kh, kw, _ = w.shape
+    Ho, Wo = (H + 2 * pad - kh) // stride + 1, (W + 2 * pad - kw) // stride + 1
+    m = np.ascontiguousarray(mask, dtype=np.uint8)
+    if m.size != Ho * Wo:
+        raise ValueError("the mask must have Ho*Wo entries")
+    b = None if bias is None else _f32(bias)
+    y = np.empty((Nb, Ho, Wo, C_out), dtype=np.float32)
+    rc = lib.asxo_alg2_fp32(_ptr(x, ctypes.c_float), Nb, H, W, C_in, _ptr(w, ctypes.c_float), C_out, kh, kw,
+                            stride, pad, None if b is None else _ptr(b, ctypes.c_float),
+                            _ptr(m, ctypes.c_uint8), int(bool(relu)), _ptr(y, ctypes.c_float))
+    if rc != 0:
+        raise ValueError("bad geometry")
     return y

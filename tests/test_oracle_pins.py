@@ -299,3 +299,30 @@ def test_generated_masks_have_the_stated_structure():
     assert len(wl.config(2)) == 20 and len(wl.config(4)) == 31 and len(wl.config(5)) == 18
     dense = sum(2 * s.M * s.K * s.N for s in wl.config(3))
     assert abs(dense / 1e9 - 232.1) < 0.2
+
+
+# ----------------------------------------------------------------------------- the paper's three stages
+@pytest.mark.parametrize("name", ["t_3x3_c64", "t_3x3_s2", "t_1x1_s2", "t_7x7_c3", "t_5x5_c24", "t_3x3_c5_n7"])
+def test_definition_equals_the_papers_three_stages_in_fp32(name):
+    """Appendix A, Algorithm 2 written out as a separate program (pointer indirection buffer over the
+    kept positions, dense product on the reduced range, reverse in-place expansion with the running
+    id) reaches the oracle's plain definition up to fp32 rounding; dropped positions are exact zeros."""
+    spec = [s for s in wl.iter_small_cases() if s.name == name][0]
+    x, w, b, m = wl.make_x(spec), wl.make_w(spec), wl.make_b(spec), wl.make_layer_mask(spec)
+    xb, wb = oracle.bf16_round(x), oracle.bf16_round(w)
+    for relu in (True, False):
+        ref = oracle.masked_conv(x, w, b, m, spec.stride, spec.pad, relu)
+        got = oracle.alg2_fp32(xb, wb, b, m, spec.stride, spec.pad, relu).astype(np.float64)
+        assert np.linalg.norm(got - ref) <= 2e-6 * np.linalg.norm(ref)
+        dropped = np.tile(m, spec.Nb).reshape(spec.Nb, spec.Ho, spec.Wo) == 0
+        assert not got[dropped].any() and not ref[dropped].any()
+
+
+def test_three_stage_expansion_handles_all_kept_and_all_dropped():
+    rng = np.random.default_rng(21)
+    x = rng.standard_normal((2, 6, 5, 4)).astype(np.float32)
+    w = rng.standard_normal((3, 3, 3, 4)).astype(np.float32)
+    for mask in (np.ones(30, np.uint8), np.zeros(30, np.uint8)):
+        ref = oracle.masked_conv(x, w, None, mask, 1, 1, False)
+        got = oracle.alg2_fp32(oracle.bf16_round(x), oracle.bf16_round(w), None, mask, 1, 1, False)
+        assert np.allclose(got, ref, rtol=1e-5, atol=1e-5)
