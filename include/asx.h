@@ -134,6 +134,18 @@ asx_status asx_set_mask_from_scores(asx_layer* layer, const float* score, int H0
 asx_status asx_set_input_mask(asx_layer* layer, const uint8_t* mask, int64_t rows, void* cuda_stream);
 
 /*
+ * Residual add in the epilogue (the shortcut of a residual block; part of chaining layers without
+ * extra passes over the activations): with a residual tensor set, asx_run computes
+ *     y = mask ? act(acc + bias + residual) : 0
+ * where `residual` is a bfloat16 tensor laid out exactly like y in that call (dense
+ * [Nb][Ho][Wo][C_out], or [Nb*P'][C_out] with ASX_OUT_COMPACT).  Only kept rows of it are read.
+ *   residual_dev : device pointer owned by the caller, aligned like y, valid during every following
+ *                  asx_run of this layer; NULL (the default) switches the add off.
+ * Not available with ASX_IMPL_NAIVE (asx_run returns ASX_ERR_INVALID_ARG).
+ */
+asx_status asx_set_residual(asx_layer* layer, const void* residual_dev);
+
+/*
  * Rebuild the kept-row list from the stored mask (stage i alone; the same work the
  * ASX_RECOMPACT flag does inside asx_run).  Asynchronous on `cuda_stream`; allocates nothing.
  * ASX_ERR_NO_MASK before any asx_set_mask*.

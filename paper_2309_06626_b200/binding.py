@@ -16,7 +16,7 @@ EXPORTS = (
     "asx_status_string", "asx_create_layer", "asx_set_mask", "asx_set_mask_random", "asx_recompact", "asx_run",
     "asx_get_kept", "asx_get_kept_host", "asx_get_mask", "asx_last_device_status", "asx_destroy",
     "asx_compact_scratch_bytes", "asx_compact", "asx_compact_status", "asx_compact_static",
-    "asx_mask_from_scores", "asx_set_mask_from_scores", "asx_mask_from_activation", "asx_set_input_mask",
+    "asx_mask_from_scores", "asx_set_mask_from_scores", "asx_mask_from_activation", "asx_set_input_mask", "asx_set_residual",
 )
 COMPACT_STATIC_MAX_ROWS = 1 << 24
 
@@ -59,6 +59,7 @@ def lib():
         L.asx_compact_status.argtypes = [vp, vp]
         L.asx_compact_static.argtypes = [vp, i64, vp, vp, vp]
         L.asx_set_input_mask.argtypes = [vp, vp, i64, vp]
+        L.asx_set_residual.argtypes = [vp, vp]
         L.asx_mask_from_activation.argtypes = [vp, i64, ci, vp, vp]
         L.asx_mask_from_scores.argtypes = [vp, ci, ci, ci, ci, ctypes.c_double, vp]
         L.asx_set_mask_from_scores.argtypes = [vp, vp, ci, ci, ci, ci, ctypes.c_double, vp]
@@ -120,6 +121,11 @@ class MaskedConvLayer:
             m = np.ascontiguousarray(mask, dtype=np.uint8)
             ptr, rows = m.ctypes.data, m.size
         _check(lib().asx_set_input_mask(self._h, ptr, rows, _stream_ptr(stream)), "asx_set_input_mask")
+
+    def set_residual(self, residual=None) -> None:
+        """CUDA bf16 tensor laid out like the output, added before the activation; None switches it off.
+        The caller keeps the tensor alive while the layer runs."""
+        _check(lib().asx_set_residual(self._h, 0 if residual is None else residual.data_ptr()), "asx_set_residual")
 
     def set_mask_random(self, rows: int, sparsity: float, block: int, seed: int, stream=None) -> None:
         _check(lib().asx_set_mask_random(self._h, rows, float(sparsity), block, seed, _stream_ptr(stream)),

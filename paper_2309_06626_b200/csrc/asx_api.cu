@@ -24,6 +24,7 @@ struct asx_layer {
     int32_t* d_small = nullptr;        // [0] kept count, [1] status word
     bool has_mask = false;
     int64_t host_kept = -1;            // kept entries of the mask when it came from the host, else -1
+    const void* residual = nullptr;    // caller-owned shortcut tensor added in the epilogue, or null
     int32_t* d_in_rank = nullptr;      // compact input: row of each input position within its image, -1 = dropped
     int64_t in_rows = 0, in_rank_cap = 0;
     int64_t in_kept = 0;
@@ -281,6 +282,13 @@ asx_status asx_set_mask_from_scores(asx_layer* L, const float* score, int H0, in
     return asx_set_mask(L, mask.data(), (int64_t)Ho * Wo, cuda_stream);
 }
 
+asx_status asx_set_residual(asx_layer* L, const void* residual_dev)
+{
+    if (L == nullptr) return ASX_ERR_INVALID_ARG;
+    L->residual = residual_dev;
+    return ASX_OK;
+}
+
 asx_status asx_set_input_mask(asx_layer* L, const uint8_t* mask, int64_t rows, void* cuda_stream)
 {
     if (L == nullptr || mask == nullptr || rows < 1 || rows >= (1ll << 31)) return ASX_ERR_INVALID_ARG;
@@ -340,7 +348,8 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     if (L == nullptr || x == nullptr || w == nullptr || y == nullptr) return ASX_ERR_INVALID_ARG;
     if (Nb < 1 || H < 1 || W < 1) return ASX_ERR_INVALID_ARG;
     if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE | ASX_OUT_COMPACT | ASX_IN_COMPACT)) return ASX_ERR_INVALID_ARG;
-    if ((flags & ASX_IMPL_NAIVE) && (flags & (ASX_OUT_COMPACT | ASX_IN_COMPACT))) return ASX_ERR_INVALID_ARG;
+    if ((flags & ASX_IMPL_NAIVE) && ((flags & (ASX_OUT_COMPACT | ASX_IN_COMPACT)) || L->residual != nullptr)) return ASX_ERR_INVALID_ARG;
+    if (L->residual != nullptr && (reinterpret_cast<uintptr_t>(L->residual) & ((L->C_out % 8 == 0) ? 15 : 1))) return ASX_ERR_ALIGN;
     if (H + 2 * L->pad < L->kh || W + 2 * L->pad < L->kw) return ASX_ERR_INVALID_ARG;
     if (!L->has_mask) return ASX_ERR_NO_MASK;
     asx_status s = bind_device(L);
@@ -559,7 +568,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     }
     return from_cuda(launch_fast(g, plan, L->tmap, plan.vec == 2 ? L->tmap_x : L->tmap, xsrc, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
                                  L->num_sms, fuse_compact ? 1 : 0, L->host_kept, static_cast<float*>(L->d_ws), L->d_wscnt,
-                                 out_compact ? 1 : 0, in_compact ? L->d_in_rank : nullptr, (int)L->in_kept, st));
+                                 out_compact ? 1 : 0, in_compact ? L->d_in_rank : nullptr, (int)L->in_kept, L->residual, st));
 }
 
 asx_status asx_get_kept(asx_layer* L, int64_t* count, const int32_t** dev_kept)

@@ -71,7 +71,7 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
                         const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
                         int num_sms, int fuse_compact, long long host_kept, float* ws_partial, int* ws_counters,
-                        int out_compact, const int32_t* in_rank, int in_kept, cudaStream_t st);
+                        int out_compact, const int32_t* in_rank, int in_kept, const void* residual, cudaStream_t st);
 // src[rows][C] -> dst[rows][Cp] with zero channels added (Cp = 4 or a multiple of 8; rows*Cp % 8 == 0)
 cudaError_t launch_pad_channels(const void* src, void* dst, long long rows, int C, int Cp, cudaStream_t st);
 // filters for the pixel-pair form: w[C_out][kh][kw][C] -> w2[C_out][kh][kw2][2][4], where pair kxx,

@@ -92,6 +92,7 @@ struct FastArgs {
     int fuse_compact;   // rebuild the kept-row list from the mask inside this kernel (small masks)
     int32_t* kept_out;  // where the fused compaction writes the list and its count
     int32_t* count_out;
+    const __nv_bfloat16* residual;   // non-null: added to acc + bias before the activation, same layout as y
     int out_compact;    // y holds the kept rows only, in kept order (row rk at y[rk][*]); nothing is zero-filled
     const int32_t* in_rank;   // non-null: x holds only the rows its own mask kept; in_rank[pos] = row of input position
                               // pos within its image's in_kept rows, or -1 for a dropped position (read as zeros)
@@ -241,6 +242,29 @@ __device__ __forceinline__ int out_row_of(int rk, const FastDiv& fdcnt, const Co
     return kept.at(rk);
 }
 
+// Eight values of the residual tensor (the shortcut branch of a residual block, laid out like the
+// output) starting at element `off`, as fp32; zeros when there is no residual.  `left` = columns left
+// in the row (only the first min(left, 8) are read on the element-wise path).
+__device__ __forceinline__ void load_residual8(const __nv_bfloat16* residual, long long off, int left, int vec, float* res)
+{
+#pragma unroll
+    for (int j = 0; j < 8; ++j) res[j] = 0.f;
+    if (residual == nullptr) return;
+    if (vec) {
+        const uint4 q = __ldg(reinterpret_cast<const uint4*>(residual + off));
+        const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            res[2 * j] = __uint_as_float(w4[j] << 16);
+            res[2 * j + 1] = __uint_as_float(w4[j] & 0xffff0000u);
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (j < left) res[j] = __bfloat162float(residual[off + j]);
+    }
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 {
     const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
@@ -297,7 +321,7 @@ __device__ __forceinline__ int2 row_info_of(int rk, int Mk, const FastDiv& fdcnt
     return info;
 }
 
-template <int MODE, bool IN_COMPACT>
+template <int MODE, bool IN_COMPACT, bool RESIDUAL>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                          const ConvGeom g, const FastArgs a)
@@ -594,6 +618,12 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                         }
                     }
                     float v[8] = {lo4.x, lo4.y, lo4.z, lo4.w, hi4.x, hi4.y, hi4.z, hi4.w};
+                    if (RESIDUAL) {
+                        float res[8];
+                        load_residual8(a.residual, yrow + n0 + gq * 8, 8, 1, res);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) v[j] += res[j];
+                    }
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const float f = v[j] + sbias[gq * 8 + j];
@@ -637,10 +667,16 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                         if (colh >= N || c0 + 8 * h >= BN) break;      // the tile's last chunk may be 16 columns wide
                         float v[8];
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            float f = __uint_as_float(r[8 * h + j]);
-                            f += sbias[c0 + 8 * h + j];
-                            v[j] = a.relu ? fmaxf(f, 0.f) : f;
+                        for (int j = 0; j < 8; ++j) v[j] = __uint_as_float(r[8 * h + j]) + sbias[c0 + 8 * h + j];
+                        if (RESIDUAL) {                        // a separate instance: even an untaken branch here costs the plain path 3 %
+                            float res[8];
+                            load_residual8(a.residual, yoff + colh, N - colh, a.vec_out, res);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) v[j] += res[j];
+                        }
+                        if (a.relu) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) v[j] = fmaxf(v[j], 0.f);
                         }
                         if (a.vec_out) {
                             uint4 o;
@@ -1043,7 +1079,7 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
                         const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
                         int num_sms, int fuse_compact, long long host_kept, float* ws_partial, int* ws_counters,
-                        int out_compact, const int32_t* in_rank, int in_kept, cudaStream_t st)
+                        int out_compact, const int32_t* in_rank, int in_kept, const void* residual, cudaStream_t st)
 {
     FastArgs a;
     a.fdcnt_host = make_fastdiv((uint32_t)(host_kept > 0 && host_kept < (1ll << 31) ? host_kept : 1));
@@ -1060,6 +1096,7 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     a.dev_status = dev_status;
     a.relu = relu;
     a.out_compact = out_compact;
+    a.residual = static_cast<const __nv_bfloat16*>(residual);
     a.in_rank = in_rank;
     a.in_kept = in_kept;
     a.BN = plan.BN;
@@ -1085,11 +1122,13 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     int grid = (int)(tiles < num_sms ? tiles : num_sms);
     if (grid < 1) grid = 1;
     const int variant = plan.vec + (in_rank != nullptr ? 2 : 0);      // 1, 2: dense input; 3, 4: compact input
-    auto kern = variant == 2   ? masked_conv_sm100_kernel<GATHER_TMA, false>
-                : variant == 1 ? masked_conv_sm100_kernel<GATHER_CPASYNC, false>
-                : variant == 4 ? masked_conv_sm100_kernel<GATHER_TMA, true>
-                               : masked_conv_sm100_kernel<GATHER_CPASYNC, true>;
-    static int smem_set[5] = {0, 0, 0, 0, 0};   // largest dynamic shared memory size enabled so far, per variant
+    const bool has_res = residual != nullptr;
+    auto kern = variant == 2   ? (has_res ? masked_conv_sm100_kernel<GATHER_TMA, false, true> : masked_conv_sm100_kernel<GATHER_TMA, false, false>)
+                : variant == 1 ? (has_res ? masked_conv_sm100_kernel<GATHER_CPASYNC, false, true> : masked_conv_sm100_kernel<GATHER_CPASYNC, false, false>)
+                : variant == 4 ? (has_res ? masked_conv_sm100_kernel<GATHER_TMA, true, true> : masked_conv_sm100_kernel<GATHER_TMA, true, false>)
+                               : (has_res ? masked_conv_sm100_kernel<GATHER_CPASYNC, true, true> : masked_conv_sm100_kernel<GATHER_CPASYNC, true, false>);
+    static int smem_set_all[10] = {0};          // largest dynamic shared memory size enabled so far, per instance
+    int* smem_set = smem_set_all + (has_res ? 5 : 0);
     if (plan.smem_bytes > smem_set[variant]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
         if (e != cudaSuccess) return e;

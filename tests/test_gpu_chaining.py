@@ -119,3 +119,55 @@ def test_compact_output_next_to_its_input_in_memory():
     layer.close()
     ref = oracle.masked_conv(x, w, b, m, 1, 1, True).reshape(spec.M, spec.C_out)[np.flatnonzero(m)]
     assert _rel(yc.float().cpu().numpy().astype(np.float64), ref) < 5e-3
+
+
+RES_CASES = [
+    # C_in, C_out, k, s, p, H, W, Nb, sparsity %, block, compact output
+    (64, 64, 3, 1, 1, 20, 23, 2, 40, 1, False),      # TMA gather, dense output
+    (16, 40, 3, 2, 1, 29, 31, 2, 50, 4, False),      # cp.async gather, 48-wide tile with a 16-column tail
+    (64, 64, 3, 1, 1, 14, 14, 3, 30, 2, True),       # compact output: the residual is compact too
+    (512, 64, 3, 1, 1, 7, 7, 4, 50, 1, False),       # few rows, long reduction: the add happens after the k shares are summed
+    (5, 7, 3, 1, 1, 12, 11, 2, 30, 1, False),        # odd channel counts: element-wise loads and stores
+]
+
+
+@pytest.mark.parametrize("case", RES_CASES, ids=[f"r{i}" for i in range(len(RES_CASES))])
+def test_residual_add_before_the_activation(case):
+    """y = mask ? relu(conv + bias + residual) : 0, the shortcut of a residual block fused into the
+    epilogue.  The oracle gives conv + bias without activation; the rest is written out here."""
+    cin, cout, k, s, p, H, W, Nb, sp, blk, compact = case
+    spec = wl.LayerSpec("res", cin, cout, k, k, s, p, H, W, Nb, sp, blk, "relu", wl.BASE_SEED + 310)
+    x, w, b, m = wl.make_x(spec), wl.make_w(spec), wl.make_b(spec), wl.make_layer_mask(spec)
+    rng = np.random.default_rng(12)
+    res = oracle.bf16_round(rng.standard_normal((spec.M, cout)).astype(np.float32)).astype(np.float64)
+    fm = np.tile(m, Nb).astype(bool)
+    lin = oracle.masked_conv(x, w, b, m, s, p, False).reshape(spec.M, cout)
+    ref = np.where(fm[:, None], np.maximum(lin + res, 0.0), 0.0)
+    rows = np.flatnonzero(fm)
+    layer = asx.MaskedConvLayer(cin, cout, k, k, s, p)
+    layer.set_mask(m)
+    xd, wd, bd = to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda()
+    if compact:
+        rd = to_dev_bf16(res[rows].astype(np.float32))
+        y = torch.full((rows.size, cout), float("nan"), dtype=torch.bfloat16, device="cuda")
+        flags = asx.ACT_RELU | asx.RECOMPACT | asx.OUT_COMPACT
+    else:
+        rd = to_dev_bf16(res.astype(np.float32))
+        y = torch.full((spec.M, cout), float("nan"), dtype=torch.bfloat16, device="cuda")
+        flags = asx.ACT_RELU | asx.RECOMPACT
+    layer.set_residual(rd)
+    st = int(torch.cuda.current_stream().cuda_stream)
+    assert layer.run_raw(xd.data_ptr(), Nb, H, W, wd.data_ptr(), bd.data_ptr(), y.data_ptr(), flags | asx.IMPL_NAIVE, st) == 1
+    _run_raw(layer, xd, Nb, H, W, wd, bd, y, flags)
+    got = y.float().cpu().numpy().astype(np.float64)
+    assert not np.isnan(got).any()
+    want = ref[rows] if compact else ref
+    assert _rel(got, want) < 5e-3
+    if not compact:
+        assert not got[~fm].any()
+    # switching the residual off gives the plain layer again
+    layer.set_residual(None)
+    _run_raw(layer, xd, Nb, H, W, wd, bd, y, flags)
+    layer.close()
+    plain = np.where(fm[:, None], np.maximum(lin, 0.0), 0.0)
+    assert _rel(y.float().cpu().numpy().astype(np.float64), plain[rows] if compact else plain) < 5e-3
