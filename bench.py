@@ -37,12 +37,12 @@ L2_BYTES = 126 * 1024 * 1024
 
 # DRAM traffic of the dominant kernel from one ncu capture of the default workload (ResNet-18 stack,
 # batch 64): dram__bytes_read.sum + dram__bytes_write.sum averaged over the 20 fused-kernel launches
-# of a step (12.17 MB read + 2.35 MB written; ncu flushes the caches before every captured launch,
+# of a step (12.18 MB read + 2.35 MB written; ncu flushes the caches before every captured launch,
 # so reads are cold-cache and most of a launch's output is still in L2 when its counters stop).
 # The figure belongs to the kernel sources whose digest is recorded with it; with any other sources
 # the bench reports null.
-NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.52e6,
-               "csrc_sha256": "0322820e2ae0d641279a704bf6806d5d026011b8ec1f7c7e8659f075cc8c6abf"}
+NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.53e6,
+               "csrc_sha256": "502c232532e7f7254845b6cafad49d19abb3fc1e71fec6361a3cd4c71eea633e"}
 
 
 def csrc_digest() -> str:
