@@ -3,7 +3,7 @@
 // Appendix A, Algorithm 2 (first function) walks the output positions in raster order and
 // appends an entry for every position whose mask is 1; the running index of that loop is an
 // exclusive prefix sum of the mask.  Here the prefix sum is a single-pass chained scan:
-// each 4096-row tile counts its kept rows (16 mask bytes per thread, popcount, a shuffle
+// each 16384-row tile counts its kept rows (4 x 16 mask bytes per thread, popcount, a shuffle
 // scan inside each warp and across the warp totals), publishes its total, and finds the
 // number of kept rows before it by looking back over its predecessors' published values,
 // 32 predecessors at a time with a warp ballot.  Tiles take their numbers from an atomic
@@ -31,13 +31,20 @@ __device__ __forceinline__ unsigned nonzero_bytes4(unsigned w)
     return ((t >> 7) & 1u) | ((t >> 14) & 2u) | ((t >> 21) & 4u) | ((t >> 28) & 8u);
 }
 
-__global__ void __launch_bounds__(COMPACT_THREADS)
+// A block takes COMPACT_SUB consecutive 4096-row sub-tiles: all their mask bytes are loaded before
+// anything else (four 16-byte loads in flight per thread instead of one: with one, the kernel was
+// bound by the latency of a tile's load -> scan -> look-back -> store chain at 1.5 TB/s), one
+// look-back serves all of them, and the index staging buffer is reused sub-tile by sub-tile.
+constexpr int COMPACT_SUB = 4;
+constexpr int COMPACT_BIG_TILE = COMPACT_SUB * COMPACT_TILE;
+
+__global__ void __launch_bounds__(COMPACT_THREADS, 8)
 compact_kernel(const uint8_t* __restrict__ mask, long long rows, int32_t* __restrict__ kept,
                int32_t* __restrict__ count, ScratchHeader* hdr,
                volatile unsigned long long* status, int num_tiles)
 {
     __shared__ int32_t s_idx[COMPACT_TILE];
-    __shared__ int s_warp_total[COMPACT_THREADS / 32];
+    __shared__ int s_warp_total[COMPACT_SUB][COMPACT_THREADS / 32];
     __shared__ int s_tile;
     __shared__ int s_exclusive;
 
@@ -49,35 +56,57 @@ compact_kernel(const uint8_t* __restrict__ mask, long long rows, int32_t* __rest
     const int tile = s_tile;
     if (tile >= num_tiles) return;
 
-    // 16 mask bytes per thread -> 16 flag bits
-    const long long first = (long long)tile * COMPACT_TILE + (long long)tid * COMPACT_PER_THREAD;
-    unsigned flags = 0;
+    // 16 mask bytes per thread and sub-tile -> 16 flag bits each
+    const long long tile_first = (long long)tile * COMPACT_BIG_TILE;
     const bool aligned = (reinterpret_cast<uintptr_t>(mask) & 15) == 0;
-    if (aligned && first + COMPACT_PER_THREAD <= rows) {
-        const uint4 v = *reinterpret_cast<const uint4*>(mask + first);
-        flags = nonzero_bytes4(v.x) | (nonzero_bytes4(v.y) << 4) | (nonzero_bytes4(v.z) << 8) |
-                (nonzero_bytes4(v.w) << 12);
-    } else {
-        for (int j = 0; j < COMPACT_PER_THREAD; ++j)
-            if (first + j < rows && mask[first + j] != 0) flags |= 1u << j;
-    }
-    const int mine = __popc(flags);
-
-    // inclusive shuffle scan inside the warp, then over the warp totals
-    int incl = mine;
+    unsigned flags[COMPACT_SUB];
+    uint4 raw[COMPACT_SUB];
+    bool fast[COMPACT_SUB];
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += t;
+    for (int sub = 0; sub < COMPACT_SUB; ++sub) {
+        const long long first = tile_first + (long long)sub * COMPACT_TILE + (long long)tid * COMPACT_PER_THREAD;
+        fast[sub] = aligned && first + COMPACT_PER_THREAD <= rows;
+        raw[sub] = make_uint4(0, 0, 0, 0);
+        if (fast[sub]) raw[sub] = *reinterpret_cast<const uint4*>(mask + first);
     }
-    if (lane == 31) s_warp_total[warp] = incl;
+    int mine[COMPACT_SUB], incl[COMPACT_SUB];
+#pragma unroll
+    for (int sub = 0; sub < COMPACT_SUB; ++sub) {
+        const long long first = tile_first + (long long)sub * COMPACT_TILE + (long long)tid * COMPACT_PER_THREAD;
+        unsigned f = 0;
+        if (fast[sub]) {
+            f = nonzero_bytes4(raw[sub].x) | (nonzero_bytes4(raw[sub].y) << 4) | (nonzero_bytes4(raw[sub].z) << 8) |
+                (nonzero_bytes4(raw[sub].w) << 12);
+        } else {
+            for (int j = 0; j < COMPACT_PER_THREAD; ++j)
+                if (first + j < rows && mask[first + j] != 0) f |= 1u << j;
+        }
+        flags[sub] = f;
+        mine[sub] = __popc(f);
+        // inclusive shuffle scan inside the warp
+        int v = mine[sub];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, v, d);
+            if (lane >= d) v += t;
+        }
+        incl[sub] = v;
+        if (lane == 31) s_warp_total[sub][warp] = v;
+    }
     __syncthreads();
-    int warp_prefix = 0, tile_total = 0;
+    int warp_prefix[COMPACT_SUB], sub_total[COMPACT_SUB], tile_total = 0;
 #pragma unroll
-    for (int i = 0; i < COMPACT_THREADS / 32; ++i) {
-        const int t = s_warp_total[i];
-        if (i < warp) warp_prefix += t;
-        tile_total += t;
+    for (int sub = 0; sub < COMPACT_SUB; ++sub) {
+        int wp = 0, tot = 0;
+#pragma unroll
+        for (int i = 0; i < COMPACT_THREADS / 32; ++i) {
+            const int t = s_warp_total[sub][i];
+            if (i < warp) wp += t;
+            tot += t;
+        }
+        warp_prefix[sub] = wp;
+        sub_total[sub] = tot;
+        tile_total += tot;
     }
 
     // chained scan across tiles
@@ -125,18 +154,25 @@ compact_kernel(const uint8_t* __restrict__ mask, long long rows, int32_t* __rest
         }
     }
 
-    // ordered write: into shared memory first, then coalesced to the list
-    int at = warp_prefix + incl - mine;
-    unsigned f = flags;
-    while (f) {
-        const int j = __ffs(f) - 1;
-        f &= f - 1;
-        s_idx[at++] = (int32_t)(first + j);
+    // ordered write, sub-tile by sub-tile: into shared memory first, then coalesced to the list
+    int base = 0;                                              // kept rows of this tile before the sub-tile
+#pragma unroll
+    for (int sub = 0; sub < COMPACT_SUB; ++sub) {
+        const long long first = tile_first + (long long)sub * COMPACT_TILE + (long long)tid * COMPACT_PER_THREAD;
+        const int at = warp_prefix[sub] + incl[sub] - mine[sub];
+        const unsigned f = flags[sub];
+        if (f) {                                               // sixteen independent predicated stores, no loop over set bits
+#pragma unroll
+            for (int j = 0; j < COMPACT_PER_THREAD; ++j)
+                if ((f >> j) & 1u) s_idx[at + __popc(f & ((1u << j) - 1u))] = (int32_t)(first + j);
+        }
+        __syncthreads();                                       // also publishes s_exclusive on the first pass
+        const int exclusive = s_exclusive + base;
+        for (int i = tid; i < sub_total[sub]; i += COMPACT_THREADS) kept[exclusive + i] = s_idx[i];
+        base += sub_total[sub];
+        __syncthreads();                                       // s_idx is reused
     }
-    __syncthreads();
-    const int exclusive = s_exclusive;
-    for (int i = tid; i < tile_total; i += COMPACT_THREADS) kept[exclusive + i] = s_idx[i];
-    if (tile == num_tiles - 1 && tid == 0) *count = exclusive + tile_total;
+    if (tile == num_tiles - 1 && tid == 0) *count = s_exclusive + tile_total;
 }
 
 // Masks of up to 16 384 rows (every per-layer mask of a classification network) need no chained
@@ -194,7 +230,7 @@ compact_small_kernel(const uint8_t* __restrict__ mask, int rows, int32_t* __rest
 
 }  // namespace
 
-static int tiles_for(int64_t rows)
+static int tiles_for(int64_t rows)      // 4096-row units: sizes the scratch (one status word each; the kernel uses every fourth)
 {
     int64_t t = (rows + COMPACT_TILE - 1) / COMPACT_TILE;
     return (int)(t < 1 ? 1 : t);
@@ -211,7 +247,7 @@ cudaError_t launch_compact(const uint8_t* mask, int64_t rows, int32_t* kept, int
     auto* hdr = static_cast<ScratchHeader*>(scratch);
     if (rows <= COMPACT_SMALL_MAX_ROWS)
         return launch_pdl(compact_small_kernel, dim3(1), dim3(1024), 0, st, mask, (int)rows, kept, count, hdr);
-    const int tiles = tiles_for(rows);
+    const int tiles = (int)((rows + COMPACT_BIG_TILE - 1) / COMPACT_BIG_TILE);
     cudaError_t e = cudaMemsetAsync(scratch, 0, (size_t)compact_scratch_bytes(rows), st);
     if (e != cudaSuccess) return e;
     auto* status = reinterpret_cast<volatile unsigned long long*>(hdr + 1);
