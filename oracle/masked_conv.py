@@ -27,7 +27,7 @@ def build(force: bool = False) -> str:
         return _LIB
     tmp = _LIB + f".tmp{os.getpid()}"
     subprocess.check_call(["gcc", "-O2", "-std=c11", "-fopenmp", "-shared", "-fPIC",
-                           "-o", tmp, _SRC, _SRC_ALG2])
+                           "-o", tmp, _SRC, _SRC_ALG2, "-lm"])
     os.replace(tmp, _LIB)
     return _LIB
 
@@ -96,10 +96,18 @@ def _geometry(x, w, stride, pad):
     return Nb, H, W, C_in, C_out, kh, kw, Ho, Wo
 
 
+def _act_code(relu) -> int:
+    """Activation code of the C oracle: False/None/"none" -> 0, True/"relu" -> 1, "silu" -> 2."""
+    if isinstance(relu, str):
+        return {"none": 0, "relu": 1, "silu": 2}[relu]
+    return int(bool(relu))
+
+
 def masked_conv(x, w, bias: Optional[np.ndarray], mask, stride: int, pad: int,
-                relu: bool) -> np.ndarray:
+                relu) -> np.ndarray:
     """y[Nb][Ho][Wo][C_out] in fp64.  x is NHWC fp32, w is [C_out][kh][kw][C_in] fp32 (both are
-    rounded to bf16 inside), bias fp32 or None, mask uint8 of Ho*Wo or Nb*Ho*Wo entries."""
+    rounded to bf16 inside), bias fp32 or None, mask uint8 of Ho*Wo or Nb*Ho*Wo entries.
+    `relu` is a bool (ReLU or identity) or one of "none", "relu", "silu"."""
     x, w = _f32(x), _f32(w)
     Nb, H, W, C_in, C_out, kh, kw, Ho, Wo = _geometry(x, w, stride, pad)
     mask = np.ascontiguousarray(mask, dtype=np.uint8).ravel()
@@ -108,13 +116,13 @@ def masked_conv(x, w, bias: Optional[np.ndarray], mask, stride: int, pad: int,
     rc = _load().asxo_masked_conv(
         _ptr(x, ctypes.c_float), Nb, H, W, C_in, _ptr(w, ctypes.c_float), C_out, kh, kw,
         stride, pad, None if b is None else _ptr(b, ctypes.c_float),
-        _ptr(mask, ctypes.c_uint8), mask.size, int(bool(relu)), _ptr(y, ctypes.c_double))
+        _ptr(mask, ctypes.c_uint8), mask.size, _act_code(relu), _ptr(y, ctypes.c_double))
     if rc:
         raise ValueError(f"oracle rejected the arguments (code {rc})")
     return y
 
 
-def masked_conv_rows(x, w, bias, mask, stride: int, pad: int, relu: bool, sel) -> np.ndarray:
+def masked_conv_rows(x, w, bias, mask, stride: int, pad: int, relu, sel) -> np.ndarray:
     """The same definition at selected lowered rows only: returns [len(sel)][C_out] fp64."""
     x, w = _f32(x), _f32(w)
     Nb, H, W, C_in, C_out, kh, kw, Ho, Wo = _geometry(x, w, stride, pad)
@@ -125,7 +133,7 @@ def masked_conv_rows(x, w, bias, mask, stride: int, pad: int, relu: bool, sel) -
     rc = _load().asxo_masked_conv_rows(
         _ptr(x, ctypes.c_float), Nb, H, W, C_in, _ptr(w, ctypes.c_float), C_out, kh, kw,
         stride, pad, None if b is None else _ptr(b, ctypes.c_float),
-        _ptr(mask, ctypes.c_uint8), mask.size, int(bool(relu)),
+        _ptr(mask, ctypes.c_uint8), mask.size, _act_code(relu),
         _ptr(sel, ctypes.c_int64), sel.size, _ptr(y, ctypes.c_double))
     if rc:
         raise ValueError(f"oracle rejected the arguments (code {rc})")

@@ -22,6 +22,9 @@
  *    out_x inner); a mask of Ho*Wo entries is shared by all images of the batch, a mask of
  *    Nb*Ho*Wo entries gives one bit per lowered row;
  *  - cross-correlation (no kernel flip), symmetric zero padding, dilation 1, groups 1;
+ *  - the activation `act` is a code: 0 identity, 1 ReLU max(z, 0), 2 SiLU z / (1 + exp(-z))
+ *    (the activation of YOLOv5, one of the networks of Section 4); both map 0 to 0, so a
+ *    dropped position equals the activation of a zero pre-activation without bias;
  *  - inputs and weights are rounded to bfloat16 (round to nearest, ties to even) first,
  *    then every product and sum is taken in double precision; the bias is an fp32 vector
  *    added before the activation; the result is NOT rounded.
@@ -31,9 +34,18 @@
  * all-ones inputs, unit impulses, hand-computed tiny integer cases, and the invariants of
  * the kept-row list.
  */
+#include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
+
+/* Activation by code, in double precision. */
+static double activate(double z, int act)
+{
+    if (act == 1) return z < 0.0 ? 0.0 : z;
+    if (act == 2) return z / (1.0 + exp(-z));
+    return z;
+}
 
 /* bfloat16 rounding, round-to-nearest-even, written out on the bit pattern. */
 static float bf16_rne(float f)
@@ -73,7 +85,7 @@ typedef struct {
 
 /* One output pixel (all channels) by the definition. */
 static void one_position(const geom_t *g, const float *xr, const float *wr, const float *bias,
-                         int relu, int n, int oy, int ox, double *y)
+                         int act, int n, int oy, int ox, double *y)
 {
     for (int co = 0; co < g->C_out; ++co) {
         double s = bias ? (double)bias[co] : 0.0;
@@ -89,8 +101,7 @@ static void one_position(const geom_t *g, const float *xr, const float *wr, cons
                     s += (double)xp[ci] * (double)wp[ci];
             }
         }
-        if (relu && s < 0.0) s = 0.0;
-        y[co] = s;
+        y[co] = activate(s, act);
     }
 }
 
@@ -112,7 +123,7 @@ static int fill_geom(geom_t *g, int Nb, int H, int W, int C_in, int C_out, int k
  * Returns 0, or 1 on bad arguments, 2 on allocation failure. */
 int asxo_masked_conv(const float *x, int Nb, int H, int W, int C_in,
                      const float *w, int C_out, int kh, int kw, int stride, int pad,
-                     const float *bias, const uint8_t *mask, int64_t rows, int relu, double *y)
+                     const float *bias, const uint8_t *mask, int64_t rows, int act, double *y)
 {
     geom_t g;
     if (fill_geom(&g, Nb, H, W, C_in, C_out, kh, kw, stride, pad)) return 1;
@@ -134,7 +145,7 @@ int asxo_masked_conv(const float *x, int Nb, int H, int W, int C_in,
                 if (!keep) {
                     for (int co = 0; co < C_out; ++co) yo[co] = 0.0;
                 } else {
-                    one_position(&g, xr, wr, bias, relu, n, oy, ox, yo);
+                    one_position(&g, xr, wr, bias, act, n, oy, ox, yo);
                 }
             }
     free(xr); free(wr);
@@ -146,7 +157,7 @@ int asxo_masked_conv(const float *x, int Nb, int H, int W, int C_in,
  * x and w must already hold bf16-representable values when pre_rounded != 0. */
 int asxo_masked_conv_rows(const float *x, int Nb, int H, int W, int C_in,
                           const float *w, int C_out, int kh, int kw, int stride, int pad,
-                          const float *bias, const uint8_t *mask, int64_t rows, int relu,
+                          const float *bias, const uint8_t *mask, int64_t rows, int act,
                           const int64_t *sel, int64_t nsel, double *y)
 {
     geom_t g;
@@ -186,8 +197,7 @@ int asxo_masked_conv_rows(const float *x, int Nb, int H, int W, int C_in,
                         s += (double)bf16_rne(xp[ci]) * (double)wp[ci];
                 }
             }
-            if (relu && s < 0.0) s = 0.0;
-            yo[co] = s;
+            yo[co] = activate(s, act);
         }
     }
     free(wr);

@@ -326,3 +326,50 @@ def test_three_stage_expansion_handles_all_kept_and_all_dropped():
         ref = oracle.masked_conv(x, w, None, mask, 1, 1, False)
         got = oracle.alg2_fp32(oracle.bf16_round(x), oracle.bf16_round(w), None, mask, 1, 1, False)
         assert np.allclose(got, ref, rtol=1e-5, atol=1e-5)
+
+
+# ---- SiLU (the activation of YOLOv5, one of the networks of Section 4)
+
+def _one_by_one(values, bias, act, mask=None):
+    """A 1x1 convolution with weight 1 over one row of pixels: the pre-activation is value + bias."""
+    x = np.asarray(values, dtype=np.float32).reshape(1, 1, -1, 1)
+    w = np.ones((1, 1, 1, 1), dtype=np.float32)
+    b = np.asarray([bias], dtype=np.float32)
+    m = np.ones(x.shape[2], dtype=np.uint8) if mask is None else np.asarray(mask, dtype=np.uint8)
+    return oracle.masked_conv(x, w, b, m, 1, 0, act).ravel()
+
+
+def test_silu_closed_forms():
+    # values exactly representable in bf16, so the pre-activation is known exactly
+    z = np.array([0.0, 0.5, 1.0, -2.0, 3.5, -8.0, 16.0, -0.25])
+    y = _one_by_one(z, 0.0, "silu")
+    import math
+    # z sigma(z) written with tanh instead of exp: sigma(z) = (1 + tanh(z / 2)) / 2
+    ref = np.array([0.5 * v * (1.0 + math.tanh(0.5 * v)) for v in z])
+    np.testing.assert_allclose(y, ref, rtol=1e-14, atol=1e-16)
+    assert y[0] == 0.0
+    # printed values of z sigma(z): 1 -> 0.7310585786..., -2 -> -0.2384058440...
+    assert abs(y[2] - 0.7310585786300049) < 1e-15
+    assert abs(y[3] + 0.2384058440442351) < 1e-15
+    # odd part: silu(z) - silu(-z) = z
+    y2 = _one_by_one(-z, 0.0, "silu")
+    np.testing.assert_allclose(y - y2, z, rtol=0, atol=1e-15)
+    # bounded below by its minimum -0.27846..., close to z for large z, close to 0 for very negative z
+    dense = _one_by_one(np.arange(-64, 64) / 8.0, 0.0, "silu")
+    assert dense.min() > -0.2785 and dense.min() < -0.278
+    assert abs(y[6] - 16.0) < 2e-6 and -3e-3 < y[5] < 0.0
+
+
+def test_silu_applies_after_bias_and_only_on_kept_positions():
+    z = np.array([1.0, -1.0, 2.0, 0.5])
+    y = _one_by_one(z, 0.5, "silu", mask=[1, 0, 1, 0])
+    import math
+    assert y[1] == 0.0 and y[3] == 0.0                       # not silu(bias)
+    for i in (0, 2):
+        v = z[i] + 0.5
+        assert abs(y[i] - v / (1.0 + math.exp(-v))) < 1e-15
+    # the three activation codes differ where they should
+    none = _one_by_one(z, 0.5, "none", mask=[1, 1, 1, 1])
+    relu = _one_by_one(z, 0.5, "relu", mask=[1, 1, 1, 1])
+    np.testing.assert_array_equal(none, z + 0.5)
+    np.testing.assert_array_equal(relu, np.maximum(z + 0.5, 0.0))
