@@ -42,7 +42,7 @@ L2_BYTES = 126 * 1024 * 1024
 # The figure belongs to the kernel sources whose digest is recorded with it; with any other sources
 # the bench reports null.
 NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.53e6,
-               "csrc_sha256": "5683e19353dd0f67860ac19d25de147fec7dfcd7f9836f521f25238d2bed9e52"}
+               "csrc_sha256": "c89186eceed59fa557e01f983450c73ac1beb2ee940b06b7a353acc0ca07b967"}
 
 
 def csrc_digest() -> str:
@@ -291,7 +291,7 @@ def run_ours(args):
     peaks = load_peaks()
     st_obj = torch.cuda.current_stream()
     st = int(st_obj.cuda_stream)
-    RELU = asx.ACT_RELU
+    RELU = asx.ACT_SILU if args.act == "silu" else asx.ACT_RELU      # the activation flag of every asx_run below
 
     specs = wl.config(args.config)
     if args.only:
@@ -600,6 +600,7 @@ def run_ours(args):
                    "step": "per layer: one asx_run with ASX_RECOMPACT = mask compaction (inside the fused kernel "
                            "for masks <= 16384 rows) + gather/GEMM/scatter"
                            + ("" if graph is None else "; one step = one CUDA-graph replay"),
+                   "activation": args.act,
                    "mask": "one mask per layer shared by the batch"
                            + ("" if args.mask == "blocks" else "; masks from one random input-resolution score, average-pooled"
                               " to each layer and ranked (Algorithm 1, getMask)")},
@@ -613,7 +614,7 @@ def run_ours(args):
                 "ms_per_step": e2e_ms},
         "gpu_launches": K * sum(L.launches for L in layers),
         "roofline": {"bound": "tensor", "kernel": "masked_conv_sm100_kernel", "achieved": achieved,
-                     "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": measured_traffic(args.config, args.only or (args.mask != "blocks")),
+                     "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": measured_traffic(args.config, args.only or (args.mask != "blocks") or (args.act != "relu")),
                      "traffic_unit": "bytes per launch (ncu dram read + write, average over the step's fused-kernel launches)",
                      "algorithmic_bytes_per_launch": sum(L.bytes for L in layers) / len(layers),
                      "peak_source": f"{peaks['source']} (sustained bf16 matmul; burst {peaks['bf16_tflops']})",
@@ -643,6 +644,8 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--act", default="relu", choices=["relu", "silu"],
+                    help="epilogue activation of every layer (silu: the YOLOv5-style variant; the headline uses relu)")
     ap.add_argument("--mask", default="blocks", choices=["blocks", "scores"],
                     help="blocks: seeded blocks of dropped rows; scores: the paper's getMask from one random score")
     ap.add_argument("--no-s1", action="store_true", help="skip the stand-alone compaction bandwidth leg")

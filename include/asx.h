@@ -55,7 +55,9 @@ enum {
     ASX_RECOMPACT = 2,     /* rebuild the kept-row list from the stored mask inside this call */
     ASX_IMPL_NAIVE = 4,    /* run the slow one-thread-per-output CUDA kernel (debug reference) */
     ASX_OUT_COMPACT = 8,   /* y holds the kept rows only: [Nb*P'][C_out] in kept order, nothing zero-filled */
-    ASX_IN_COMPACT = 16    /* x holds only the positions kept by the mask given to asx_set_input_mask */
+    ASX_IN_COMPACT = 16,   /* x holds only the positions kept by the mask given to asx_set_input_mask */
+    ASX_ACT_SILU = 32      /* y = z / (1 + exp(-z)), z = acc + bias, on kept rows (the activation of the YOLOv5
+                              network of Section 4); not together with ASX_ACT_RELU (ASX_ERR_INVALID_ARG) */
 };
 
 /* Human-readable name of a status code; never NULL; static storage. */
@@ -161,7 +163,8 @@ asx_status asx_recompact(asx_layer* layer, void* cuda_stream);
  *   bias : device, fp32 [C_out], 4-byte aligned, or NULL for zero bias.
  *   y    : device, bf16 [Nb][Ho][Wo][C_out], Ho = (H + 2*pad - kh)/stride + 1 (Wo alike);
  *          16-byte aligned when C_out % 8 == 0, else 2-byte; must not overlap x.
- *   flags: OR of ASX_ACT_RELU, ASX_RECOMPACT, ASX_IMPL_NAIVE, ASX_OUT_COMPACT, ASX_IN_COMPACT.  With
+ *   flags: OR of ASX_ACT_RELU or ASX_ACT_SILU, ASX_RECOMPACT, ASX_IMPL_NAIVE, ASX_OUT_COMPACT, ASX_IN_COMPACT.
+ *          Dropped positions are 0 under every activation (each maps 0 to 0; no bias is added there).  With
  *          ASX_OUT_COMPACT y is bf16 [Nb*P'][C_out] (P' = kept entries of the mask, which must then be
  *          shared by the batch); with ASX_IN_COMPACT x is bf16 [Nb*P'_in][C_in] (see asx_set_input_mask).
  * Asynchronous on `cuda_stream`.  Allocates in two cases only, on first use and when the buffers

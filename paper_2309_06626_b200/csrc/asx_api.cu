@@ -347,7 +347,8 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
 {
     if (L == nullptr || x == nullptr || w == nullptr || y == nullptr) return ASX_ERR_INVALID_ARG;
     if (Nb < 1 || H < 1 || W < 1) return ASX_ERR_INVALID_ARG;
-    if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE | ASX_OUT_COMPACT | ASX_IN_COMPACT)) return ASX_ERR_INVALID_ARG;
+    if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE | ASX_OUT_COMPACT | ASX_IN_COMPACT | ASX_ACT_SILU)) return ASX_ERR_INVALID_ARG;
+    if ((flags & ASX_ACT_RELU) && (flags & ASX_ACT_SILU)) return ASX_ERR_INVALID_ARG;      // one activation at most
     if ((flags & ASX_IMPL_NAIVE) && ((flags & (ASX_OUT_COMPACT | ASX_IN_COMPACT)) || L->residual != nullptr)) return ASX_ERR_INVALID_ARG;
     if (L->residual != nullptr && (reinterpret_cast<uintptr_t>(L->residual) & ((L->C_out % 8 == 0) ? 15 : 1))) return ASX_ERR_ALIGN;
     if (H + 2 * L->pad < L->kh || W + 2 * L->pad < L->kw) return ASX_ERR_INVALID_ARG;
@@ -401,7 +402,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         s = run_compaction(L, st);
         if (s != ASX_OK) return s;
     }
-    const int relu = (flags & ASX_ACT_RELU) ? 1 : 0;
+    const int relu = (flags & ASX_ACT_SILU) ? 2 : (flags & ASX_ACT_RELU) ? 1 : 0;      // activation code: 0 identity, 1 ReLU, 2 SiLU
     int32_t* d_count = L->d_small;
     int* d_status = reinterpret_cast<int*>(L->d_small + 1);
 

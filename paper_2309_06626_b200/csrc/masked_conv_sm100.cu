@@ -265,6 +265,13 @@ __device__ __forceinline__ void load_residual8(const __nv_bfloat16* residual, lo
     }
 }
 
+// z * sigmoid(z) with the fast exponential and division (relative error about 1e-6, far below the
+// bf16 rounding of the result); exp(-z) = inf for very negative z gives -0.
+__device__ __forceinline__ float silu(float z)
+{
+    return __fdividef(z, 1.f + __expf(-z));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 {
     const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
@@ -321,7 +328,9 @@ __device__ __forceinline__ int2 row_info_of(int rk, int Mk, const FastDiv& fdcnt
     return info;
 }
 
-template <int MODE, bool IN_COMPACT, bool RESIDUAL>
+// SILU: the activation is z / (1 + exp(-z)) instead of the run-time choice between ReLU and identity
+// (an instance of its own, like RESIDUAL: the plain path pays for every extra branch in the epilogue).
+template <int MODE, bool IN_COMPACT, bool RESIDUAL, bool SILU>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                          const ConvGeom g, const FastArgs a)
@@ -627,7 +636,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const float f = v[j] + sbias[gq * 8 + j];
-                        v[j] = a.relu ? fmaxf(f, 0.f) : f;
+                        v[j] = SILU ? silu(f) : a.relu ? fmaxf(f, 0.f) : f;
                     }
                     uint4 o;
                     o.x = pack_bf16(v[0], v[1]);
@@ -674,7 +683,10 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
 #pragma unroll
                             for (int j = 0; j < 8; ++j) v[j] += res[j];
                         }
-                        if (a.relu) {
+                        if (SILU) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) v[j] = silu(v[j]);
+                        } else if (a.relu) {
 #pragma unroll
                             for (int j = 0; j < 8; ++j) v[j] = fmaxf(v[j], 0.f);
                         }
@@ -1094,7 +1106,7 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     a.kept = kept;
     a.count = count;
     a.dev_status = dev_status;
-    a.relu = relu;
+    a.relu = relu == 1 ? 1 : 0;
     a.out_compact = out_compact;
     a.residual = static_cast<const __nv_bfloat16*>(residual);
     a.in_rank = in_rank;
@@ -1122,13 +1134,19 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     int grid = (int)(tiles < num_sms ? tiles : num_sms);
     if (grid < 1) grid = 1;
     const int variant = plan.vec + (in_rank != nullptr ? 2 : 0);      // 1, 2: dense input; 3, 4: compact input
-    const bool has_res = residual != nullptr;
-    auto kern = variant == 2   ? (has_res ? masked_conv_sm100_kernel<GATHER_TMA, false, true> : masked_conv_sm100_kernel<GATHER_TMA, false, false>)
-                : variant == 1 ? (has_res ? masked_conv_sm100_kernel<GATHER_CPASYNC, false, true> : masked_conv_sm100_kernel<GATHER_CPASYNC, false, false>)
-                : variant == 4 ? (has_res ? masked_conv_sm100_kernel<GATHER_TMA, true, true> : masked_conv_sm100_kernel<GATHER_TMA, true, false>)
-                               : (has_res ? masked_conv_sm100_kernel<GATHER_CPASYNC, true, true> : masked_conv_sm100_kernel<GATHER_CPASYNC, true, false>);
-    static int smem_set_all[10] = {0};          // largest dynamic shared memory size enabled so far, per instance
-    int* smem_set = smem_set_all + (has_res ? 5 : 0);
+    const bool has_res = residual != nullptr, is_silu = relu == 2;
+    using Kern = void (*)(const CUtensorMap, const CUtensorMap, const ConvGeom, const FastArgs);
+    Kern kern = nullptr;
+#define ASX_PICK(MODE, IC)                                                                                          \
+    kern = has_res ? (is_silu ? masked_conv_sm100_kernel<MODE, IC, true, true> : masked_conv_sm100_kernel<MODE, IC, true, false>) \
+                   : (is_silu ? masked_conv_sm100_kernel<MODE, IC, false, true> : masked_conv_sm100_kernel<MODE, IC, false, false>)
+    if (variant == 2) { ASX_PICK(GATHER_TMA, false); }
+    else if (variant == 1) { ASX_PICK(GATHER_CPASYNC, false); }
+    else if (variant == 4) { ASX_PICK(GATHER_TMA, true); }
+    else { ASX_PICK(GATHER_CPASYNC, true); }
+#undef ASX_PICK
+    static int smem_set_all[20] = {0};          // largest dynamic shared memory size enabled so far, per instance
+    int* smem_set = smem_set_all + (has_res ? 5 : 0) + (is_silu ? 10 : 0);
     if (plan.smem_bytes > smem_set[variant]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
         if (e != cudaSuccess) return e;

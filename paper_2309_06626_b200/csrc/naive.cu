@@ -57,7 +57,8 @@ __global__ void naive_kept_rows(ConvGeom g, const __nv_bfloat16* __restrict__ x,
             }
         }
         float v = acc + (bias ? bias[co] : 0.f);
-        if (relu) v = fmaxf(v, 0.f);
+        if (relu == 1) v = fmaxf(v, 0.f);
+        if (relu == 2) v = v / (1.f + expf(-v));     // SiLU
         y[(long long)row * g.C_out + co] = __float2bfloat16_rn(v);
     }
 }

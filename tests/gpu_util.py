@@ -47,7 +47,7 @@ def full_row_mask(spec, mask):
 
 def check_against_oracle(spec, x, w, b, mask, flags, rows_sel=None):
     """Full comparison (rows_sel None) or comparison on selected lowered rows."""
-    relu = bool(flags & asx.ACT_RELU)
+    relu = "silu" if flags & asx.ACT_SILU else bool(flags & asx.ACT_RELU)      # the oracle's activation argument
     y, bits, kept = run_library(spec, x, w, b, mask, flags, prefill=0x7fc1)   # NaN canary
     # kept list: bit-exact
     assert np.array_equal(kept, oracle.kept_list(mask)), "kept-row list differs"

@@ -131,18 +131,21 @@ RES_CASES = [
 ]
 
 
+@pytest.mark.parametrize("act", ["relu", "silu"])
 @pytest.mark.parametrize("case", RES_CASES, ids=[f"r{i}" for i in range(len(RES_CASES))])
-def test_residual_add_before_the_activation(case):
-    """y = mask ? relu(conv + bias + residual) : 0, the shortcut of a residual block fused into the
+def test_residual_add_before_the_activation(case, act):
+    """y = mask ? act(conv + bias + residual) : 0, the shortcut of a residual block fused into the
     epilogue.  The oracle gives conv + bias without activation; the rest is written out here."""
     cin, cout, k, s, p, H, W, Nb, sp, blk, compact = case
+    act_flag = asx.ACT_RELU if act == "relu" else asx.ACT_SILU
+    f = (lambda z: np.maximum(z, 0.0)) if act == "relu" else (lambda z: z / (1.0 + np.exp(-z)))
     spec = wl.LayerSpec("res", cin, cout, k, k, s, p, H, W, Nb, sp, blk, "relu", wl.BASE_SEED + 310)
     x, w, b, m = wl.make_x(spec), wl.make_w(spec), wl.make_b(spec), wl.make_layer_mask(spec)
     rng = np.random.default_rng(12)
     res = oracle.bf16_round(rng.standard_normal((spec.M, cout)).astype(np.float32)).astype(np.float64)
     fm = np.tile(m, Nb).astype(bool)
     lin = oracle.masked_conv(x, w, b, m, s, p, False).reshape(spec.M, cout)
-    ref = np.where(fm[:, None], np.maximum(lin + res, 0.0), 0.0)
+    ref = np.where(fm[:, None], f(lin + res), 0.0)
     rows = np.flatnonzero(fm)
     layer = asx.MaskedConvLayer(cin, cout, k, k, s, p)
     layer.set_mask(m)
@@ -150,11 +153,11 @@ def test_residual_add_before_the_activation(case):
     if compact:
         rd = to_dev_bf16(res[rows].astype(np.float32))
         y = torch.full((rows.size, cout), float("nan"), dtype=torch.bfloat16, device="cuda")
-        flags = asx.ACT_RELU | asx.RECOMPACT | asx.OUT_COMPACT
+        flags = act_flag | asx.RECOMPACT | asx.OUT_COMPACT
     else:
         rd = to_dev_bf16(res.astype(np.float32))
         y = torch.full((spec.M, cout), float("nan"), dtype=torch.bfloat16, device="cuda")
-        flags = asx.ACT_RELU | asx.RECOMPACT
+        flags = act_flag | asx.RECOMPACT
     layer.set_residual(rd)
     st = int(torch.cuda.current_stream().cuda_stream)
     assert layer.run_raw(xd.data_ptr(), Nb, H, W, wd.data_ptr(), bd.data_ptr(), y.data_ptr(), flags | asx.IMPL_NAIVE, st) == 1
@@ -169,5 +172,5 @@ def test_residual_add_before_the_activation(case):
     layer.set_residual(None)
     _run_raw(layer, xd, Nb, H, W, wd, bd, y, flags)
     layer.close()
-    plain = np.where(fm[:, None], np.maximum(lin, 0.0), 0.0)
+    plain = np.where(fm[:, None], f(lin), 0.0)
     assert _rel(y.float().cpu().numpy().astype(np.float64), plain[rows] if compact else plain) < 5e-3

@@ -64,6 +64,45 @@ def test_tiny_integer_cases_bit_exact(k, p, impl):
             assert np.array_equal(kept, oracle.kept_list(mask))
 
 
+@pytest.mark.parametrize("impl", IMPLS, ids=[i[0] for i in IMPLS])
+@pytest.mark.parametrize("spec", SMALL, ids=[s.name for s in SMALL])
+def test_small_cases_silu(spec, impl):
+    """The SiLU epilogue (own kernel instances) on every small case, split-K layers included."""
+    x, w, b, mask = make_problem(spec)
+    check_against_oracle(spec, x, w, b, mask, asx.ACT_SILU | impl[1])
+
+
+def test_silu_values_on_exact_preactivations():
+    """1x1, weight 1, inputs exact in bf16: the pre-activation is x + bias exactly, so the output
+    is bf16(silu(x + bias)) up to the error of the fast exponential (well inside half a bf16 ulp
+    except at rounding ties, hence one ulp allowed)."""
+    vals = np.array([0.0, 0.5, 1.0, -2.0, 3.5, -8.0, 16.0, -0.25, -40.0, 40.0, -100.0, 6.0], dtype=np.float32)
+    spec = wl.LayerSpec("silu1x1", 8, 8, 1, 1, 1, 0, 3, 4, 1, 0, 1, "relu", 1)
+    x = np.zeros((1, 3, 4, 8), np.float32)
+    x[0, :, :, 0] = vals.reshape(3, 4)
+    w = np.zeros((8, 1, 1, 8), np.float32)
+    w[:, 0, 0, 0] = 1.0
+    b = np.full(8, 0.5, np.float32)
+    mask = np.ones(12, np.uint8)
+    mask[5] = 0
+    y, bits, kept = run_library(spec, x, w, b, mask, asx.ACT_SILU, prefill=0x7fc1)
+    ref = oracle.masked_conv(x, w, b, mask, 1, 0, "silu").reshape(12, 8)
+    assert not np.any(bits[5])
+    ulp = np.maximum(np.abs(ref), 2.0 ** -126) * 2.0 ** -7
+    assert np.all(np.abs(y - ref) <= ulp), np.abs(y - ref).max()
+    assert np.all(np.isfinite(y))
+
+
+def test_relu_and_silu_together_are_rejected():
+    layer = asx.MaskedConvLayer(8, 8, 1, 1, 1, 0)
+    layer.set_mask(np.ones(4, np.uint8))
+    x = torch.zeros((1, 2, 2, 8), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((8, 1, 1, 8), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(asx.AsxError):
+        layer.run(x, w, None, flags=asx.ACT_RELU | asx.ACT_SILU)
+    layer.close()
+
+
 def test_all_dropped_ignores_nan_input():
     spec = wl.LayerSpec("nan", 8, 16, 3, 3, 1, 1, 9, 9, 2, 100, 1, "relu", 7)
     x, w, b, _ = make_problem(spec)
