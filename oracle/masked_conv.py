@@ -96,18 +96,19 @@ def _geometry(x, w, stride, pad):
     return Nb, H, W, C_in, C_out, kh, kw, Ho, Wo
 
 
-def _act_code(relu) -> int:
-    """Activation code of the C oracle: False/None/"none" -> 0, True/"relu" -> 1, "silu" -> 2."""
-    if isinstance(relu, str):
-        return {"none": 0, "relu": 1, "silu": 2}[relu]
-    return int(bool(relu))
+def _act_code(relu, storage: str = "bf16") -> int:
+    """Activation code of the C oracle: False/None/"none" -> 0, True/"relu" -> 1, "silu" -> 2;
+    plus 16 for fp32 storage (x and w taken as given instead of being rounded to bf16)."""
+    code = {"none": 0, "relu": 1, "silu": 2}[relu] if isinstance(relu, str) else int(bool(relu))
+    return code + {"bf16": 0, "fp32": 16}[storage]
 
 
 def masked_conv(x, w, bias: Optional[np.ndarray], mask, stride: int, pad: int,
-                relu) -> np.ndarray:
+                relu, storage: str = "bf16") -> np.ndarray:
     """y[Nb][Ho][Wo][C_out] in fp64.  x is NHWC fp32, w is [C_out][kh][kw][C_in] fp32 (both are
     rounded to bf16 inside), bias fp32 or None, mask uint8 of Ho*Wo or Nb*Ho*Wo entries.
-    `relu` is a bool (ReLU or identity) or one of "none", "relu", "silu"."""
+    `relu` is a bool (ReLU or identity) or one of "none", "relu", "silu"; storage="fp32" keeps x and w
+    as given (the paper's fp32 storage) instead of rounding them to bf16."""
     x, w = _f32(x), _f32(w)
     Nb, H, W, C_in, C_out, kh, kw, Ho, Wo = _geometry(x, w, stride, pad)
     mask = np.ascontiguousarray(mask, dtype=np.uint8).ravel()
@@ -116,13 +117,13 @@ def masked_conv(x, w, bias: Optional[np.ndarray], mask, stride: int, pad: int,
     rc = _load().asxo_masked_conv(
         _ptr(x, ctypes.c_float), Nb, H, W, C_in, _ptr(w, ctypes.c_float), C_out, kh, kw,
         stride, pad, None if b is None else _ptr(b, ctypes.c_float),
-        _ptr(mask, ctypes.c_uint8), mask.size, _act_code(relu), _ptr(y, ctypes.c_double))
+        _ptr(mask, ctypes.c_uint8), mask.size, _act_code(relu, storage), _ptr(y, ctypes.c_double))
     if rc:
         raise ValueError(f"oracle rejected the arguments (code {rc})")
     return y
 
 
-def masked_conv_rows(x, w, bias, mask, stride: int, pad: int, relu, sel) -> np.ndarray:
+def masked_conv_rows(x, w, bias, mask, stride: int, pad: int, relu, sel, storage: str = "bf16") -> np.ndarray:
     """The same definition at selected lowered rows only: returns [len(sel)][C_out] fp64."""
     x, w = _f32(x), _f32(w)
     Nb, H, W, C_in, C_out, kh, kw, Ho, Wo = _geometry(x, w, stride, pad)
@@ -133,7 +134,7 @@ def masked_conv_rows(x, w, bias, mask, stride: int, pad: int, relu, sel) -> np.n
     rc = _load().asxo_masked_conv_rows(
         _ptr(x, ctypes.c_float), Nb, H, W, C_in, _ptr(w, ctypes.c_float), C_out, kh, kw,
         stride, pad, None if b is None else _ptr(b, ctypes.c_float),
-        _ptr(mask, ctypes.c_uint8), mask.size, _act_code(relu),
+        _ptr(mask, ctypes.c_uint8), mask.size, _act_code(relu, storage),
         _ptr(sel, ctypes.c_int64), sel.size, _ptr(y, ctypes.c_double))
     if rc:
         raise ValueError(f"oracle rejected the arguments (code {rc})")

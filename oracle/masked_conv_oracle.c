@@ -25,6 +25,8 @@
  *  - the activation `act` is a code: 0 identity, 1 ReLU max(z, 0), 2 SiLU z / (1 + exp(-z))
  *    (the activation of YOLOv5, one of the networks of Section 4); both map 0 to 0, so a
  *    dropped position equals the activation of a zero pre-activation without bias;
+ *  - adding 16 to the activation code selects fp32 storage (the paper's, Appendix A: sizeof(float)):
+ *    inputs and weights are then taken as given instead of being rounded to bfloat16;
  *  - inputs and weights are rounded to bfloat16 (round to nearest, ties to even) first,
  *    then every product and sum is taken in double precision; the bias is an fp32 vector
  *    added before the activation; the result is NOT rounded.
@@ -133,8 +135,14 @@ int asxo_masked_conv(const float *x, int Nb, int H, int W, int C_in,
     float *xr = (float *)malloc(sizeof(float) * (size_t)nx);
     float *wr = (float *)malloc(sizeof(float) * (size_t)nw);
     if (!xr || !wr) { free(xr); free(wr); return 2; }
-    asxo_bf16_round(x, xr, nx);
-    asxo_bf16_round(w, wr, nw);
+    if (act & 16) {                       /* fp32 storage: the values as given */
+        memcpy(xr, x, sizeof(float) * (size_t)nx);
+        memcpy(wr, w, sizeof(float) * (size_t)nw);
+    } else {
+        asxo_bf16_round(x, xr, nx);
+        asxo_bf16_round(w, wr, nw);
+    }
+    act &= 15;
 #pragma omp parallel for collapse(2) schedule(dynamic, 1)
     for (int n = 0; n < Nb; ++n)
         for (int oy = 0; oy < g.Ho; ++oy)
@@ -167,7 +175,10 @@ int asxo_masked_conv_rows(const float *x, int Nb, int H, int W, int C_in,
     const int64_t nw = (int64_t)C_out * kh * kw * C_in;
     float *wr = (float *)malloc(sizeof(float) * (size_t)nw);
     if (!wr) return 2;
-    asxo_bf16_round(w, wr, nw);
+    const int exact = (act & 16) != 0;    /* fp32 storage: the values as given */
+    act &= 15;
+    if (exact) memcpy(wr, w, sizeof(float) * (size_t)nw);
+    else asxo_bf16_round(w, wr, nw);
     int bad = 0;
 #pragma omp parallel for schedule(dynamic, 4)
     for (int64_t i = 0; i < nsel; ++i) {
@@ -194,7 +205,7 @@ int asxo_masked_conv_rows(const float *x, int Nb, int H, int W, int C_in,
                     const float *xp = x + (((int64_t)n * H + iy) * W + ix) * C_in;
                     const float *wp = wr + (((int64_t)co * kh + ky) * kw + kx) * C_in;
                     for (int ci = 0; ci < C_in; ++ci)
-                        s += (double)bf16_rne(xp[ci]) * (double)wp[ci];
+                        s += (double)(exact ? xp[ci] : bf16_rne(xp[ci])) * (double)wp[ci];
                 }
             }
             yo[co] = activate(s, act);

@@ -373,3 +373,28 @@ def test_silu_applies_after_bias_and_only_on_kept_positions():
     relu = _one_by_one(z, 0.5, "relu", mask=[1, 1, 1, 1])
     np.testing.assert_array_equal(none, z + 0.5)
     np.testing.assert_array_equal(relu, np.maximum(z + 0.5, 0.0))
+
+
+# ---- fp32 storage (the paper's, Appendix A): inputs taken as given
+
+def test_fp32_storage_equals_library_fp64_conv_on_unrounded_inputs():
+    rng = np.random.default_rng(77)
+    x = rng.standard_normal((2, 6, 7, 5)).astype(np.float32)
+    w = rng.standard_normal((4, 3, 3, 5)).astype(np.float32)
+    b = rng.standard_normal(4).astype(np.float32)
+    m = (rng.random(42) < 0.6).astype(np.uint8)
+    y = oracle.masked_conv(x, w, b, m, 1, 1, False, storage="fp32")
+    ref = torch.nn.functional.conv2d(torch.from_numpy(x).double().permute(0, 3, 1, 2),
+                                     torch.from_numpy(w).double().permute(0, 3, 1, 2),
+                                     torch.from_numpy(b).double(), padding=1).permute(0, 2, 3, 1).numpy()
+    ref = ref * np.tile(m, 2).reshape(2, 6, 7, 1)
+    np.testing.assert_allclose(y, ref, rtol=0, atol=1e-13)
+    # the inputs are not bf16 values, so the bf16-storage result must differ (the option does something)
+    assert np.abs(oracle.masked_conv(x, w, b, m, 1, 1, False) - y).max() > 1e-3
+    # on bf16-representable inputs both storages agree exactly
+    xr, wr = oracle.bf16_round(x), oracle.bf16_round(w)
+    np.testing.assert_array_equal(oracle.masked_conv(xr, wr, b, m, 1, 1, True, storage="fp32"),
+                                  oracle.masked_conv(x, w, b, m, 1, 1, True))
+    sel = np.array([0, 5, 41, 42, 80])
+    np.testing.assert_array_equal(oracle.masked_conv_rows(x, w, b, m, 1, 1, "silu", sel, storage="fp32"),
+                                  oracle.masked_conv(x, w, b, m, 1, 1, "silu", storage="fp32").reshape(84, 4)[sel])
