@@ -232,18 +232,19 @@ def run_reference(args):
 # --------------------------------------------------------------------------------------------
 # the GPU leg
 class DeviceLayer:
-    def __init__(self, spec, torch, asx, dense_twin=True, score=None):
+    def __init__(self, spec, torch, asx, dense_twin=True, score=None, f32=False):
         self.spec = spec
+        dt = torch.float32 if f32 else torch.bfloat16          # storage type of x, w and y
         x, w, b = wl.make_x(spec), wl.make_w(spec), wl.make_b(spec)
         # masks: seeded blocks of rows (default), or the paper's generator from one input-resolution score
         self.mask = (wl.make_layer_mask(spec) if score is None
                      else asx.mask_from_scores(score, spec.Ho, spec.Wo, spec.sparsity_pct / 100.0))
-        self.x_host = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+        self.x_host = torch.from_numpy(x).to(dt).pin_memory()
         self.x = self.x_host.cuda()
-        self.w = torch.from_numpy(w).to(torch.bfloat16).cuda()
+        self.w = torch.from_numpy(w).to(dt).cuda()
         self.b = torch.from_numpy(b).cuda()
-        self.y = torch.empty((spec.Nb, spec.Ho, spec.Wo, spec.C_out), dtype=torch.bfloat16, device="cuda")
-        self.y_host = torch.empty(self.y.shape, dtype=torch.bfloat16).pin_memory()
+        self.y = torch.empty((spec.Nb, spec.Ho, spec.Wo, spec.C_out), dtype=dt, device="cuda")
+        self.y_host = torch.empty(self.y.shape, dtype=dt).pin_memory()
         self.layer = asx.MaskedConvLayer(spec.C_in, spec.C_out, spec.kh, spec.kw, spec.stride, spec.pad)
         self.layer.set_mask(self.mask)
         self.dense = None
@@ -254,12 +255,12 @@ class DeviceLayer:
         self.kept_rows = kept_rows
         self.flops = wl.algorithmic_flops(spec, kept_rows)
         self.flops_dense = wl.algorithmic_flops(spec, spec.M)
-        self.bytes = wl.algorithmic_bytes(spec, self.mask)
+        self.bytes = wl.algorithmic_bytes(spec, self.mask, 4 if f32 else 2)
         self.ptrs = (self.x.data_ptr(), spec.Nb, spec.H, spec.W, self.w.data_ptr(), self.b.data_ptr(),
                      self.y.data_ptr())
         # fused kernel (it rebuilds the kept-row list itself for masks of up to 16384 rows, else a
         # compaction kernel runs first), plus channel padding of x and w when C_in % 8 != 0
-        self.launches = 1 + (0 if self.mask.size <= 16384 else 1) + (2 if spec.C_in % 8 else 0)
+        self.launches = 1 + (0 if self.mask.size <= 16384 else 1) + (2 if spec.C_in % (4 if f32 else 8) else 0)
 
     def step(self, st, flags, layer=None):
         L = layer or self.layer
@@ -291,7 +292,15 @@ def run_ours(args):
     peaks = load_peaks()
     st_obj = torch.cuda.current_stream()
     st = int(st_obj.cuda_stream)
-    RELU = asx.ACT_SILU if args.act == "silu" else asx.ACT_RELU      # the activation flag of every asx_run below
+    f32 = args.dtype == "f32"
+    # the activation (and storage) flags of every asx_run below
+    RELU = (asx.ACT_SILU if args.act == "silu" else asx.ACT_RELU) | (asx.F32 if f32 else 0)
+    if f32:
+        # fp32 storage, TF32 contraction: no measured TF32 peak exists, so the bf16 figures are scaled by
+        # the nominal dense ratio of the two tensor-core rates (1.1 / 2.25 PFLOP/s)
+        ratio = 1.1 / 2.25
+        peaks = dict(peaks, bf16_tflops=peaks["bf16_tflops"] * ratio,
+                     bf16_tflops_sustained=peaks["bf16_tflops_sustained"] * ratio)
 
     specs = wl.config(args.config)
     if args.only:
@@ -301,7 +310,7 @@ def run_ours(args):
     score = None
     if args.mask == "scores":
         score = wl.make_score(args.config, max(s.H for s in specs), max(s.W for s in specs))
-    layers = [DeviceLayer(s, torch, asx, dense_twin=(args.config != 5), score=score) for s in specs]
+    layers = [DeviceLayer(s, torch, asx, dense_twin=(args.config != 5), score=score, f32=f32) for s in specs]
     torch.cuda.synchronize()
     footprint = sum(L.x.numel() * 2 + L.y.numel() * 2 + L.w.numel() * 2 for L in layers)
 
@@ -402,7 +411,7 @@ def run_ours(args):
     cudnn_ms = None
     if rank == 0 and not args.no_cudnn:
         import torch.nn.functional as F
-        views = [(L.x.permute(0, 3, 1, 2), L.w.permute(0, 3, 1, 2), L.b.to(torch.bfloat16), L.spec) for L in layers]
+        views = [(L.x.permute(0, 3, 1, 2), L.w.permute(0, 3, 1, 2), L.b.to(L.x.dtype), L.spec) for L in layers]
 
         def cudnn_step():
             for xv, wv, bv, s in views:
@@ -420,8 +429,8 @@ def run_ours(args):
 
     # ---- end to end: host buffers, H2D of every layer's input and D2H of every output inside the timed region
     Ke = max(3, min(K, 10))
-    h2d = sum(L.x_host.numel() * 2 for L in layers)
-    d2h = sum(L.y_host.numel() * 2 for L in layers)
+    h2d = sum(L.x_host.numel() * L.x_host.element_size() for L in layers)
+    d2h = sum(L.y_host.numel() * L.y_host.element_size() for L in layers)
 
     # Copies in, kernels and copies out run on three streams, ordered per layer by events, so that the
     # two directions of the host link and the kernels overlap across layers and steps; every step still
@@ -534,7 +543,7 @@ def run_ours(args):
     chain = None
     pair = [L for L in layers if L.spec.kh == 3 and L.spec.stride == 1 and L.spec.C_in == L.spec.C_out
             and L.spec.C_in % 8 == 0 and L.mask.size == L.spec.P]
-    if not args.no_s1 and len(pair) >= 2 and pair[0].spec.H == pair[1].spec.H and pair[0].spec.C_in == pair[1].spec.C_in:
+    if not args.no_s1 and not f32 and len(pair) >= 2 and pair[0].spec.H == pair[1].spec.H and pair[0].spec.C_in == pair[1].spec.C_in:
         A, B = pair[0], pair[1]
         sa = A.spec
         kept_a, kept_b = int(A.mask.sum()), int(B.mask.sum())
@@ -592,7 +601,7 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": K,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "vs_baseline": None, "dtype": "tf32" if f32 else "bf16", "data": "synthetic",
         "config": {"workload": workload_name(args.config) + (f" [only {args.only}]" if args.only else ""),
                    "layers": len(layers),
                    "l2": f"inputs larger than L2: each step cycles {footprint / 1e6:.0f} MB of distinct "
@@ -601,6 +610,7 @@ def run_ours(args):
                            "for masks <= 16384 rows) + gather/GEMM/scatter"
                            + ("" if graph is None else "; one step = one CUDA-graph replay"),
                    "activation": args.act,
+                   "storage": "fp32 (TF32 contraction)" if f32 else "bf16",
                    "mask": "one mask per layer shared by the batch"
                            + ("" if args.mask == "blocks" else "; masks from one random input-resolution score, average-pooled"
                               " to each layer and ranked (Algorithm 1, getMask)")},
@@ -614,10 +624,11 @@ def run_ours(args):
                 "ms_per_step": e2e_ms},
         "gpu_launches": K * sum(L.launches for L in layers),
         "roofline": {"bound": "tensor", "kernel": "masked_conv_sm100_kernel", "achieved": achieved,
-                     "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": measured_traffic(args.config, args.only or (args.mask != "blocks") or (args.act != "relu")),
+                     "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf, "traffic": measured_traffic(args.config, args.only or (args.mask != "blocks") or (args.act != "relu") or f32),
                      "traffic_unit": "bytes per launch (ncu dram read + write, average over the step's fused-kernel launches)",
                      "algorithmic_bytes_per_launch": sum(L.bytes for L in layers) / len(layers),
-                     "peak_source": f"{peaks['source']} (sustained bf16 matmul; burst {peaks['bf16_tflops']})",
+                     "peak_source": f"{peaks['source']} (sustained bf16 matmul; burst {peaks['bf16_tflops']:.1f})"
+                                    + (" x 1.1/2.25, the nominal ratio of the dense TF32 and bf16 rates" if f32 else ""),
                      "kernel_ms_per_step": kern_ms,
                      "frac_of_layer_roofs": roof_ms / kern_ms,
                      "layer_roofs_ms_per_step": roof_ms},
@@ -646,6 +657,8 @@ def main():
     ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--act", default="relu", choices=["relu", "silu"],
                     help="epilogue activation of every layer (silu: the YOLOv5-style variant; the headline uses relu)")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"],
+                    help="storage of x, w and y: bf16, or fp32 (the paper's storage; the contraction then runs in TF32)")
     ap.add_argument("--mask", default="blocks", choices=["blocks", "scores"],
                     help="blocks: seeded blocks of dropped rows; scores: the paper's getMask from one random score")
     ap.add_argument("--no-s1", action="store_true", help="skip the stand-alone compaction bandwidth leg")

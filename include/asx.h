@@ -56,8 +56,10 @@ enum {
     ASX_IMPL_NAIVE = 4,    /* run the slow one-thread-per-output CUDA kernel (debug reference) */
     ASX_OUT_COMPACT = 8,   /* y holds the kept rows only: [Nb*P'][C_out] in kept order, nothing zero-filled */
     ASX_IN_COMPACT = 16,   /* x holds only the positions kept by the mask given to asx_set_input_mask */
-    ASX_ACT_SILU = 32      /* y = z / (1 + exp(-z)), z = acc + bias, on kept rows (the activation of the YOLOv5
+    ASX_ACT_SILU = 32,     /* y = z / (1 + exp(-z)), z = acc + bias, on kept rows (the activation of the YOLOv5
                               network of Section 4); not together with ASX_ACT_RELU (ASX_ERR_INVALID_ARG) */
+    ASX_F32 = 64           /* x, w and y are fp32, the storage type of Appendix A, Algorithm 2 (its sizeof(float));
+                              the products run on the tensor cores in TF32, see asx_run */
 };
 
 /* Human-readable name of a status code; never NULL; static storage. */
@@ -163,10 +165,17 @@ asx_status asx_recompact(asx_layer* layer, void* cuda_stream);
  *   bias : device, fp32 [C_out], 4-byte aligned, or NULL for zero bias.
  *   y    : device, bf16 [Nb][Ho][Wo][C_out], Ho = (H + 2*pad - kh)/stride + 1 (Wo alike);
  *          16-byte aligned when C_out % 8 == 0, else 2-byte; must not overlap x.
- *   flags: OR of ASX_ACT_RELU or ASX_ACT_SILU, ASX_RECOMPACT, ASX_IMPL_NAIVE, ASX_OUT_COMPACT, ASX_IN_COMPACT.
+ *   flags: OR of ASX_ACT_RELU or ASX_ACT_SILU, ASX_RECOMPACT, ASX_IMPL_NAIVE, ASX_OUT_COMPACT, ASX_IN_COMPACT, ASX_F32.
  *          Dropped positions are 0 under every activation (each maps 0 to 0; no bias is added there).  With
  *          ASX_OUT_COMPACT y is bf16 [Nb*P'][C_out] (P' = kept entries of the mask, which must then be
  *          shared by the batch); with ASX_IN_COMPACT x is bf16 [Nb*P'_in][C_in] (see asx_set_input_mask).
+ *          With ASX_F32 x, w and y are fp32 with the same shapes (16-byte aligned when the channel
+ *          count is a multiple of 4, else 4-byte; channel counts that are not are zero-padded to one
+ *          in layer-owned copies).  The tensor cores then read each operand as TF32: sign, exponent
+ *          and the upper 10 mantissa bits, the lower 13 bits are ignored (so inputs whose lower 13
+ *          mantissa bits are zero are multiplied exactly); sums, bias and activation are fp32 and y is
+ *          written unrounded.  ASX_IMPL_NAIVE with ASX_F32 multiplies the full fp32 values.  Not
+ *          together with ASX_OUT_COMPACT, ASX_IN_COMPACT or a residual (ASX_ERR_UNSUPPORTED).
  * Asynchronous on `cuda_stream`.  Allocates in two cases only, on first use and when the buffers
  * must grow: when C_in % 8 != 0 the layer keeps copies of x and w with the channels zero-padded to
  * a multiple of 8 (refreshed by a small kernel on every call); and when a layer has far fewer

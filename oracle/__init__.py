@@ -4,8 +4,8 @@ Only the tests, the smoke check and the benchmark's CPU-baseline leg import this
 It shares no code with the CUDA path and never imports it.
 """
 from .masked_conv import (alg2_fp32, build, bf16_round, kept_list, masked_conv, masked_conv_rows,
-                          n_threads)
+                          n_threads, tf32_operand)
 from .get_mask import get_mask, mask_from_activation, pooled_score
 
-__all__ = ["alg2_fp32", "build", "bf16_round", "kept_list", "masked_conv", "masked_conv_rows", "n_threads",
+__all__ = ["alg2_fp32", "build", "bf16_round", "kept_list", "masked_conv", "masked_conv_rows", "n_threads", "tf32_operand",
            "get_mask", "mask_from_activation", "pooled_score"]

@@ -78,6 +78,15 @@ def bf16_round(a) -> np.ndarray:
     return out
 
 
+def tf32_operand(a) -> np.ndarray:
+    """The value a TF32 tensor-core contraction uses for an fp32 operand: sign, exponent and the
+    upper 10 mantissa bits; the lower 13 mantissa bits are dropped (towards zero).  Returned as fp32.
+    For the fp32-storage path (Appendix A stores fp32): oracle result = masked_conv(tf32_operand(x),
+    tf32_operand(w), ..., storage="fp32")."""
+    a = _f32(a)
+    return (a.view(np.uint32) & np.uint32(0xFFFFE000)).view(np.float32)
+
+
 def kept_list(mask) -> np.ndarray:
     """Ascending positions with mask == 1, int32."""
     mask = np.ascontiguousarray(mask, dtype=np.uint8).ravel()

@@ -6,7 +6,7 @@ package does not load the library; the first call does, and fails loudly if the 
 has not been built.
 """
 from .binding import (AsxError, MaskedConvLayer, compact_mask, mask_from_scores, mask_from_activation, lib, lib_path, EXPORTS,
-                      ACT_RELU, RECOMPACT, IMPL_NAIVE, OUT_COMPACT, IN_COMPACT, ACT_SILU)
+                      ACT_RELU, RECOMPACT, IMPL_NAIVE, OUT_COMPACT, IN_COMPACT, ACT_SILU, F32)
 
 __all__ = ["AsxError", "MaskedConvLayer", "compact_mask", "mask_from_scores", "mask_from_activation", "lib", "lib_path", "EXPORTS",
-           "ACT_RELU", "RECOMPACT", "IMPL_NAIVE", "OUT_COMPACT", "IN_COMPACT", "ACT_SILU"]
+           "ACT_RELU", "RECOMPACT", "IMPL_NAIVE", "OUT_COMPACT", "IN_COMPACT", "ACT_SILU", "F32"]

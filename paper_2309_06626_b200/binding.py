@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libasx.so")
 _lib = None
 
-ACT_RELU, RECOMPACT, IMPL_NAIVE, OUT_COMPACT, IN_COMPACT, ACT_SILU = 1, 2, 4, 8, 16, 32
+ACT_RELU, RECOMPACT, IMPL_NAIVE, OUT_COMPACT, IN_COMPACT, ACT_SILU, F32 = 1, 2, 4, 8, 16, 32, 64
 
 # every symbol include/asx.h declares
 EXPORTS = (
@@ -147,10 +147,11 @@ class MaskedConvLayer:
     def run(self, x, w, bias=None, out=None, flags: int = ACT_RELU, stream=None):
         """x: CUDA bf16 [Nb][H][W][C_in]; w: CUDA bf16 [C_out][kh][kw][C_in]; bias: CUDA fp32 or
         None.  Returns the CUDA bf16 output [Nb][Ho][Wo][C_out] (allocated by torch unless
-        `out` is given)."""
+        `out` is given).  With the F32 flag x, w and the output are float32 instead."""
         import torch
-        if x.dtype != torch.bfloat16 or w.dtype != torch.bfloat16:
-            raise TypeError("x and w must be bfloat16")
+        dt = torch.float32 if flags & F32 else torch.bfloat16
+        if x.dtype != dt or w.dtype != dt:
+            raise TypeError("x and w must be float32 with the F32 flag, else bfloat16")
         if not (x.is_cuda and w.is_cuda and x.is_contiguous() and w.is_contiguous()):
             raise ValueError("x and w must be contiguous CUDA tensors")
         Nb, H, W, C = x.shape
@@ -158,8 +159,8 @@ class MaskedConvLayer:
             raise ValueError("tensor shapes do not match the layer")
         Ho, Wo = self.out_hw(H, W)
         if out is None:
-            out = torch.empty((Nb, Ho, Wo, self.C_out), dtype=torch.bfloat16, device=x.device)
-        elif tuple(out.shape) != (Nb, Ho, Wo, self.C_out) or out.dtype != torch.bfloat16 or not out.is_contiguous():
+            out = torch.empty((Nb, Ho, Wo, self.C_out), dtype=dt, device=x.device)
+        elif tuple(out.shape) != (Nb, Ho, Wo, self.C_out) or out.dtype != dt or not out.is_contiguous():
             raise ValueError("bad output tensor")
         bptr = 0
         if bias is not None:

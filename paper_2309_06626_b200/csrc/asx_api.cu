@@ -41,6 +41,7 @@ struct asx_layer {
     CUtensorMap tmap;
     const void* tmap_ptr = nullptr;
     int tmap_BN = 0, tmap_Kw = 0;
+    int tmap_es = 0, tmapx_es = 0;     // element size the cached tensor maps were encoded for
     CUtensorMap tmap_x;                // x as a [pixels][C_in] matrix, for the TMA row gather
     const void* tmapx_ptr = nullptr;
     int64_t tmapx_pixels = 0;
@@ -347,7 +348,12 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
 {
     if (L == nullptr || x == nullptr || w == nullptr || y == nullptr) return ASX_ERR_INVALID_ARG;
     if (Nb < 1 || H < 1 || W < 1) return ASX_ERR_INVALID_ARG;
-    if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE | ASX_OUT_COMPACT | ASX_IN_COMPACT | ASX_ACT_SILU)) return ASX_ERR_INVALID_ARG;
+    if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE | ASX_OUT_COMPACT | ASX_IN_COMPACT | ASX_ACT_SILU | ASX_F32)) return ASX_ERR_INVALID_ARG;
+    const bool f32 = (flags & ASX_F32) != 0;
+    const int ES = f32 ? 4 : 2;                 // bytes per element of x, w and y
+    const int EPC = 16 / ES;                    // elements per 16-byte chunk
+    // fp32 storage runs on dense tensors without a fused shortcut
+    if (f32 && ((flags & (ASX_OUT_COMPACT | ASX_IN_COMPACT)) || L->residual != nullptr)) return ASX_ERR_UNSUPPORTED;
     if ((flags & ASX_ACT_RELU) && (flags & ASX_ACT_SILU)) return ASX_ERR_INVALID_ARG;      // one activation at most
     if ((flags & ASX_IMPL_NAIVE) && ((flags & (ASX_OUT_COMPACT | ASX_IN_COMPACT)) || L->residual != nullptr)) return ASX_ERR_INVALID_ARG;
     if (L->residual != nullptr && (reinterpret_cast<uintptr_t>(L->residual) & ((L->C_out % 8 == 0) ? 15 : 1))) return ASX_ERR_ALIGN;
@@ -378,17 +384,17 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     }
     const int64_t x_rows = in_compact ? (int64_t)Nb * L->in_kept : (int64_t)Nb * H * W;     // rows of x in memory
 
-    const bool vec_in = (L->C_in % 8 == 0);
-    const uintptr_t in_align = vec_in ? 15 : 1;
+    const bool vec_in = (L->C_in % EPC == 0);
+    const uintptr_t in_align = vec_in ? 15 : (uintptr_t)(ES - 1);
     if ((reinterpret_cast<uintptr_t>(x) & in_align) || (reinterpret_cast<uintptr_t>(w) & in_align))
         return ASX_ERR_ALIGN;
-    if (reinterpret_cast<uintptr_t>(y) & ((L->C_out % 8 == 0) ? 15 : 1)) return ASX_ERR_ALIGN;
+    if (reinterpret_cast<uintptr_t>(y) & ((L->C_out % EPC == 0) ? 15 : (uintptr_t)(ES - 1))) return ASX_ERR_ALIGN;
     if (bias != nullptr && (reinterpret_cast<uintptr_t>(bias) & 3)) return ASX_ERR_ALIGN;
     {
-        const uintptr_t xb = reinterpret_cast<uintptr_t>(x), xe = xb + (uintptr_t)x_rows * L->C_in * 2;
+        const uintptr_t xb = reinterpret_cast<uintptr_t>(x), xe = xb + (uintptr_t)x_rows * L->C_in * ES;
         // a compact output holds Nb * P' rows (P' is known on the host for a mask that came from the host)
         const int64_t y_rows = (out_compact && L->host_kept >= 0) ? (int64_t)Nb * L->host_kept : M;
-        const uintptr_t yb = reinterpret_cast<uintptr_t>(y), ye = yb + (uintptr_t)y_rows * L->C_out * 2;
+        const uintptr_t yb = reinterpret_cast<uintptr_t>(y), ye = yb + (uintptr_t)y_rows * L->C_out * ES;
         if (xb < ye && yb < xe) return ASX_ERR_INVALID_ARG;
     }
 
@@ -407,7 +413,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     int* d_status = reinterpret_cast<int*>(L->d_small + 1);
 
     if (flags & ASX_IMPL_NAIVE)
-        return from_cuda(launch_naive(g, x, w, bias, y, L->d_mask, L->d_kept, d_count, relu, st));
+        return from_cuda(launch_naive(g, x, w, bias, y, L->d_mask, L->d_kept, d_count, relu, f32 ? 1 : 0, st));
 
     // Channel counts that are not a multiple of 8 are padded with zero channels in staging
     // copies of x and w (a filter tap of a pixel is then a whole number of 16-byte chunks); the
@@ -425,7 +431,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     // a view whose rows are 32 bytes apart (rows overlap; the borders make every tap in bounds).
     // shift = pad & 1 aligns the window to the blocks; the filter gets zero rows / columns there.
     const int bshift = L->pad & 1;
-    const bool blocks2x2 = !in_compact && L->C_in <= 4 && L->stride == 2 && (W % 2) == 0 && (H % 2) == 0 &&
+    const bool blocks2x2 = !f32 && !in_compact && L->C_in <= 4 && L->stride == 2 && (W % 2) == 0 && (H % 2) == 0 &&
                            (L->kw + bshift + 1) / 2 == 4 && L->kh + bshift <= 32;
     if (blocks2x2) {
         const int kh2 = (L->kh + bshift + 1) / 2;
@@ -466,7 +472,38 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         g.stride = 1; g.stride_w = 1;
         g.pad = 0; g.pad_w = 0;
         x_row_stride = 32;
-    } else if (L->C_in % 8 != 0) {
+    } else if (f32 && L->C_in % 4 != 0) {
+        // fp32 storage: zero channels up to a multiple of 4 (one 16-byte chunk); the padding kernel
+        // moves 2-byte units, so an fp32 tensor goes through it as twice as many of those.
+        const int Cp = (L->C_in + 3) / 4 * 4;
+        const int64_t pixels = (int64_t)Nb * H * W, taps = (int64_t)L->C_out * L->kh * L->kw;
+        if (pixels * Cp > lim) return ASX_ERR_UNSUPPORTED;
+        const size_t need_x = (size_t)pixels * Cp * 4, need_w = (size_t)taps * Cp * 4;
+        if (need_x > L->xpad_bytes || need_w > L->wpack_bytes) {
+            cudaStreamSynchronize(st);
+            if (need_x > L->xpad_bytes) {
+                cudaFree(L->d_xpad);
+                L->d_xpad = nullptr; L->xpad_bytes = 0;
+                if (cudaMalloc(&L->d_xpad, need_x) != cudaSuccess) return ASX_ERR_OOM;
+                L->xpad_bytes = need_x;
+            }
+            if (need_w > L->wpack_bytes) {
+                cudaFree(L->d_wpack);
+                L->d_wpack = nullptr; L->wpack_bytes = 0;
+                if (cudaMalloc(&L->d_wpack, need_w) != cudaSuccess) return ASX_ERR_OOM;
+                L->wpack_bytes = need_w;
+            }
+            L->tmap_ptr = nullptr;
+            L->tmapx_ptr = nullptr;
+        }
+        cudaError_t e = launch_pad_channels(x, L->d_xpad, pixels, 2 * L->C_in, 2 * Cp, st);
+        if (e == cudaSuccess) e = launch_pad_channels(w, L->d_wpack, taps, 2 * L->C_in, 2 * Cp, st);
+        if (e != cudaSuccess) return from_cuda(e);
+        xsrc = L->d_xpad;
+        wsrc = L->d_wpack;
+        g.C_in = Cp;
+        g.K = L->kh * L->kw * Cp;
+    } else if (!f32 && L->C_in % 8 != 0) {
         // Pixel-pair form for tiny channel counts under stride 2 (a network's first layer): pad the
         // channels to 4 and read two horizontally adjacent pixels as one 8-channel pixel.  The
         // convolution then has ceil((kw + shift) / 2) horizontal taps, horizontal stride 1 and left
@@ -517,8 +554,8 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     if (L->host_kept >= 0) est_rows = (L->rows == P) ? L->host_kept * Nb : L->host_kept;
     // Sharing a tile's k-blocks between blocks needs the exact tile count (to size the workspace)
     // and 16-byte output stores.
-    const bool allow_split = L->host_kept >= 0 && L->C_out % 8 == 0 && (reinterpret_cast<uintptr_t>(y) & 15) == 0;
-    if (!plan_fast(g, L->num_sms, est_rows, fuse_compact ? (int)L->rows : 0, allow_split, &plan)) return ASX_ERR_UNSUPPORTED;
+    const bool allow_split = !f32 && L->host_kept >= 0 && L->C_out % 8 == 0 && (reinterpret_cast<uintptr_t>(y) & 15) == 0;
+    if (!plan_fast(g, L->num_sms, est_rows, fuse_compact ? (int)L->rows : 0, allow_split, ES, &plan)) return ASX_ERR_UNSUPPORTED;
     if (plan.ksplit > 1) {
         const size_t need = (size_t)plan.ws_items * 128 * (size_t)plan.BN * sizeof(float);
         if (need > L->ws_bytes) {
@@ -537,39 +574,41 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         }
     }
     const int Kw = g.K;
-    if (L->tmap_ptr != wsrc || L->tmap_BN != plan.BN || L->tmap_Kw != Kw) {
+    const CUtensorMapDataType tm_type = f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const cuuint32_t box_k = (cuuint32_t)(128 / ES);           // one 128-byte swizzled row of K elements
+    if (L->tmap_ptr != wsrc || L->tmap_BN != plan.BN || L->tmap_Kw != Kw || L->tmap_es != ES) {
         EncodeTiledFn enc = encode_tiled_fn();
         if (enc == nullptr) return ASX_ERR_CUDA;
         const cuuint64_t dims[2] = {(cuuint64_t)Kw, (cuuint64_t)L->C_out};
-        const cuuint64_t strides[1] = {(cuuint64_t)Kw * 2};
-        const cuuint32_t box[2] = {64u, (cuuint32_t)plan.BN};
+        const cuuint64_t strides[1] = {(cuuint64_t)Kw * ES};
+        const cuuint32_t box[2] = {box_k, (cuuint32_t)plan.BN};
         const cuuint32_t estr[2] = {1u, 1u};
-        const CUresult r = enc(&L->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(wsrc), dims,
+        const CUresult r = enc(&L->tmap, tm_type, 2, const_cast<void*>(wsrc), dims,
                                strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return ASX_ERR_CUDA;
-        L->tmap_ptr = wsrc; L->tmap_BN = plan.BN; L->tmap_Kw = Kw;
+        L->tmap_ptr = wsrc; L->tmap_BN = plan.BN; L->tmap_Kw = Kw; L->tmap_es = ES;
     }
     if (plan.vec == 2) {
         const int64_t pixels = in_compact ? x_rows : (int64_t)Nb * g.H * g.W;
-        const int row_stride = x_row_stride ? x_row_stride : g.C_in * 2;
-        if (L->tmapx_ptr != xsrc || L->tmapx_pixels != pixels || L->tmapx_stride != row_stride) {
+        const int row_stride = x_row_stride ? x_row_stride : g.C_in * ES;
+        if (L->tmapx_ptr != xsrc || L->tmapx_pixels != pixels || L->tmapx_stride != row_stride || L->tmapx_es != ES) {
             EncodeTiledFn enc = encode_tiled_fn();
             if (enc == nullptr) return ASX_ERR_CUDA;
             const cuuint64_t dims[2] = {(cuuint64_t)g.C_in, (cuuint64_t)pixels};
             const cuuint64_t strides[1] = {(cuuint64_t)row_stride};
-            const cuuint32_t box[2] = {64u, 1u};
+            const cuuint32_t box[2] = {box_k, 1u};
             const cuuint32_t estr[2] = {1u, 1u};
-            const CUresult r = enc(&L->tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(xsrc), dims,
+            const CUresult r = enc(&L->tmap_x, tm_type, 2, const_cast<void*>(xsrc), dims,
                                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return ASX_ERR_CUDA;
-            L->tmapx_ptr = xsrc; L->tmapx_pixels = pixels; L->tmapx_stride = row_stride;
+            L->tmapx_ptr = xsrc; L->tmapx_pixels = pixels; L->tmapx_stride = row_stride; L->tmapx_es = ES;
         }
     }
     return from_cuda(launch_fast(g, plan, L->tmap, plan.vec == 2 ? L->tmap_x : L->tmap, xsrc, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
                                  L->num_sms, fuse_compact ? 1 : 0, L->host_kept, static_cast<float*>(L->d_ws), L->d_wscnt,
-                                 out_compact ? 1 : 0, in_compact ? L->d_in_rank : nullptr, (int)L->in_kept, L->residual, st));
+                                 out_compact ? 1 : 0, in_compact ? L->d_in_rank : nullptr, (int)L->in_kept, L->residual, f32 ? 1 : 0, st));
 }
 
 asx_status asx_get_kept(asx_layer* L, int64_t* count, const int32_t** dev_kept)

@@ -52,7 +52,7 @@ cudaError_t launch_compact(const uint8_t* mask, int64_t rows, int32_t* kept, int
 
 // ---- debug reference kernels (naive.cu)
 cudaError_t launch_naive(const ConvGeom& g, const void* x, const void* w, const float* bias, void* y,
-                         const uint8_t* mask, const int32_t* kept, const int32_t* count, int relu,
+                         const uint8_t* mask, const int32_t* kept, const int32_t* count, int relu, int f32,
                          cudaStream_t st);
 
 // ---- the tensor-core path (masked_conv_sm100.cu)
@@ -61,17 +61,20 @@ struct FastPlan {
     int n_tiles;      // ceil(C_out / BN)
     int stages;
     int smem_bytes;
-    int vec;          // gather mode: 1 cp.async 16 B (C_in % 8 == 0), 2 TMA row gather (C_in % 64 == 0)
-    int Kpad;         // K rounded up to 64
+    int vec;          // gather mode: 1 cp.async 16 B (a pixel's channels are whole 16-byte chunks), 2 TMA row
+                      // gather (they are whole 128-byte runs)
+    int Kpad;         // K rounded up to a whole number of stages
     int ksplit;       // work items per output tile (shares of the k-blocks); > 1 needs the workspace
     long long ws_items;   // m_tiles * n_tiles * ksplit for the estimated kept rows
 };
-bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fused_list_rows, bool allow_split, FastPlan* plan);
+// elem_bytes: 2 (bf16 storage) or 4 (fp32 storage, TF32 contraction)
+bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fused_list_rows, bool allow_split, int elem_bytes,
+               FastPlan* plan);
 cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorMap& tmap_w,
                         const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
                         int num_sms, int fuse_compact, long long host_kept, float* ws_partial, int* ws_counters,
-                        int out_compact, const int32_t* in_rank, int in_kept, const void* residual, cudaStream_t st);
+                        int out_compact, const int32_t* in_rank, int in_kept, const void* residual, int f32, cudaStream_t st);
 // src[rows][C] -> dst[rows][Cp] with zero channels added (Cp = 4 or a multiple of 8; rows*Cp % 8 == 0)
 cudaError_t launch_pad_channels(const void* src, void* dst, long long rows, int C, int Cp, cudaStream_t st);
 // filters for the pixel-pair form: w[C_out][kh][kw][C] -> w2[C_out][kh][kw2][2][4], where pair kxx,

@@ -330,7 +330,9 @@ __device__ __forceinline__ int2 row_info_of(int rk, int Mk, const FastDiv& fdcnt
 
 // SILU: the activation is z / (1 + exp(-z)) instead of the run-time choice between ReLU and identity
 // (an instance of its own, like RESIDUAL: the plain path pays for every extra branch in the epilogue).
-template <int MODE, bool IN_COMPACT, bool RESIDUAL, bool SILU>
+// F32: x, w and y are fp32 (the storage type of Appendix A); a pipeline stage is still 128 rows of
+// 128 bytes, i.e. 32 K-elements, and the tensor core reads the operands as TF32.
+template <int MODE, bool IN_COMPACT, bool RESIDUAL, bool SILU, bool F32>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                          const ConvGeom g, const FastArgs a)
@@ -349,7 +351,10 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     Shared* sh = reinterpret_cast<Shared*>(smem_raw + (smem_base - ptx::smem_u32(smem_raw)) + S * stage_bytes);
     volatile int* abort_flag = &sh->abort;
 
-    const int KB = (g.K + BK - 1) / BK;
+    constexpr int BKE = F32 ? 32 : BK;      // K elements per stage
+    constexpr int ES = F32 ? 4 : 2;         // bytes per element of x, w and y
+    constexpr int EPC = 16 / ES;            // elements per 16-byte chunk
+    const int KB = (g.K + BKE - 1) / BKE;
 
     // The layer's mask is only ever written by stream-ordered copies, never by a kernel, so the
     // fused compaction may read it while the preceding kernel is still running; the read is
@@ -449,7 +454,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                     if (!wait_bar<40>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
                     const uint32_t full = ptx::smem_u32(&sh->full[s]);
                     ptx::mbar_arrive_expect_tx(full, (uint32_t)(BN * BK * 2 + (MODE == GATHER_TMA ? A_STAGE_BYTES : 0)));
-                    ptx::tma_load_2d(smem_base + s * stage_bytes + A_STAGE_BYTES, &tmap_w, full, kb * BK, n_tile * BN);
+                    ptx::tma_load_2d(smem_base + s * stage_bytes + A_STAGE_BYTES, &tmap_w, full, kb * BKE, n_tile * BN);
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
             }
@@ -483,7 +488,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         // The whole warp runs the loop so that descriptors and counters stay in uniform registers;
         // one elected lane issues the tcgen05 instructions (issuing from inside a divergent
         // single-lane branch costs about 100 cycles per instruction).
-        const uint32_t idesc = ptx::umma_idesc_bf16(BM, BN);
+        const uint32_t idesc = F32 ? ptx::umma_idesc_tf32(BM, BN) : ptx::umma_idesc_bf16(BM, BN);
         const uint64_t adesc0 = ptx::umma_desc_k_major_sw128(smem_base);
         int s = 0, ti = 0;
         uint32_t ph = 0;
@@ -507,10 +512,17 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                 const uint64_t adesc = adesc0 + (uint64_t)(s * (stage_bytes >> 4));   // start-address field
                 const uint64_t bdesc = adesc + (A_STAGE_BYTES >> 4);
                 if (ptx::elect_one()) {
-                    ptx::umma_bf16(d, adesc, bdesc, idesc, kb != item.kb_lo ? 1u : 0u);       // 16 K-elements = 32 bytes
-                    ptx::umma_bf16(d, adesc + 2, bdesc + 2, idesc, 1u);             //   = 2 descriptor units
-                    ptx::umma_bf16(d, adesc + 4, bdesc + 4, idesc, 1u);
-                    ptx::umma_bf16(d, adesc + 6, bdesc + 6, idesc, 1u);
+                    if (F32) {                                                          // 8 K-elements = 32 bytes
+                        ptx::umma_tf32(d, adesc, bdesc, idesc, kb != item.kb_lo ? 1u : 0u);
+                        ptx::umma_tf32(d, adesc + 2, bdesc + 2, idesc, 1u);
+                        ptx::umma_tf32(d, adesc + 4, bdesc + 4, idesc, 1u);
+                        ptx::umma_tf32(d, adesc + 6, bdesc + 6, idesc, 1u);
+                    } else {
+                        ptx::umma_bf16(d, adesc, bdesc, idesc, kb != item.kb_lo ? 1u : 0u);       // 16 K-elements = 32 bytes
+                        ptx::umma_bf16(d, adesc + 2, bdesc + 2, idesc, 1u);             //   = 2 descriptor units
+                        ptx::umma_bf16(d, adesc + 4, bdesc + 4, idesc, 1u);
+                        ptx::umma_bf16(d, adesc + 6, bdesc + 6, idesc, 1u);
+                    }
                     ptx::umma_commit(ptx::smem_u32(&sh->empty[s]));
                 }
                 __syncwarp();
@@ -546,7 +558,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             if (!warp_wait_bar<100>(ptx::smem_u32(&sh->acc_full[buf]), use, abort_flag, a.dev_status)) { ok = false; break; }
             ptx::tc_fence_after_sync();
             const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
-            if (a.ksplit > 1) {
+            if (!F32 && a.ksplit > 1) {
                 // ---- split K: this item holds a partial sum.  Every share writes its partial tile
                 // to the workspace; when all shares of the tile are there, each share adds up the
                 // partials of its slice of the tile's rows, always in share order (so the result
@@ -690,7 +702,17 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
 #pragma unroll
                             for (int j = 0; j < 8; ++j) v[j] = fmaxf(v[j], 0.f);
                         }
-                        if (a.vec_out) {
+                        if (F32) {
+                            float* yf = reinterpret_cast<float*>(a.y) + yoff + colh;
+                            if (a.vec_out) {                   // C_out % 4 == 0: the row ends on a 16-byte boundary
+                                *reinterpret_cast<float4*>(yf) = make_float4(v[0], v[1], v[2], v[3]);
+                                if (colh + 4 < N) *reinterpret_cast<float4*>(yf + 4) = make_float4(v[4], v[5], v[6], v[7]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    if (colh + j < N) yf[j] = v[j];
+                            }
+                        } else if (a.vec_out) {
                             uint4 o;
                             o.x = pack_bf16(v[0], v[1]);
                             o.y = pack_bf16(v[2], v[3]);
@@ -720,12 +742,12 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         // one 16-byte column of the row and walks down the rows with a constant stride, so a warp
         // writes whole consecutive rows; four mask bytes are fetched before the four stores they
         // guard, and nothing in the loop divides.
-        unsigned short* y2 = reinterpret_cast<unsigned short*>(a.y);
+        uint8_t* yb = reinterpret_cast<uint8_t*>(a.y);
         const long long lo = (long long)g.M * blockIdx.x / gridDim.x;
         const long long hi = (long long)g.M * (blockIdx.x + 1) / gridDim.x;
         constexpr int ZT = NUM_ZERO_WARPS * 32;
         const int zt = (warp - WARP_ZERO0) * 32 + lane;
-        const int cpr = N >> 3;                                   // 16-byte chunks per row
+        const int cpr = N / EPC;                                  // 16-byte chunks per row
         const bool shared_mask = (g.rows == g.P);
         if (a.vec_out && cpr <= ZT && ZT % cpr == 0) {
             const int rpp = ZT / cpr;                             // rows covered by one pass of all threads
@@ -733,7 +755,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             long long row = lo + sub;
             int p = shared_mask ? (int)(row % g.P) : 0;           // mask index of `row`, kept incrementally
             const int pstep = rpp % g.P;
-            uint4* dst = reinterpret_cast<uint4*>(y2 + row * N + cc * 8);
+            uint4* dst = reinterpret_cast<uint4*>(yb + (row * N + cc * EPC) * ES);
             const long long dstep = (long long)rpp * cpr;         // in 16-byte units
             while (row < hi) {
                 bool drop[4];
@@ -760,9 +782,11 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                 if (__ldg(a.mask + pm) != 0) continue;
                 if (a.vec_out) {
                     for (int c1 = lane; c1 < cpr; c1 += 32)
-                        *reinterpret_cast<uint4*>(y2 + row * N + c1 * 8) = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4*>(yb + (row * N + c1 * EPC) * ES) = make_uint4(0, 0, 0, 0);
+                } else if (F32) {
+                    for (int c1 = lane; c1 < N; c1 += 32) reinterpret_cast<float*>(yb)[row * N + c1] = 0.f;
                 } else {
-                    for (int c1 = lane; c1 < N; c1 += 32) y2[row * N + c1] = 0;
+                    for (int c1 = lane; c1 < N; c1 += 32) reinterpret_cast<unsigned short*>(yb)[row * N + c1] = 0;
                 }
             }
         }
@@ -776,7 +800,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
         // bound by how fast one warp gets through an iteration, hence the two groups.
         const int pw = warp - WARP_PROD0;
         const int grp = pw / GROUP_WARPS, pwg = pw - grp * GROUP_WARPS;
-        const unsigned short* x2 = reinterpret_cast<const unsigned short*>(a.x);
+        const uint8_t* xb = reinterpret_cast<const uint8_t*>(a.x);
         if (MODE == GATHER_TMA) {
             // Lanes 0..3 of each warp run the loop on their own: each fetches four rows per stage
             // with one TMA row gather (one 64-channel slice of one filter tap per stage; padding
@@ -800,8 +824,8 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                     const Item item = item_of(t, KB, a);
                     int ky = 0, kx = 0, ci = 0;
                     if (item.kb_lo != 0) {                 // a later k share starts inside the window
-                        const int tap = item.kb_lo * BK / g.C_in;
-                        ci = item.kb_lo * BK - tap * g.C_in;
+                        const int tap = item.kb_lo * BKE / g.C_in;
+                        ci = item.kb_lo * BKE - tap * g.C_in;
                         ky = tap / g.kw;
                         kx = tap - ky * g.kw;
                     }
@@ -824,7 +848,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                             ptx::tma_gather4_2d(smem_base + s * stage_bytes + (uint32_t)(16 * pwg + 4 * lane) * 128u, &tmap_x,
                                                 ptx::smem_u32(&sh->full[s]), ci, idx[0], idx[1], idx[2], idx[3]);
                         }
-                        ci += BK;                          // next 64 channels, or the next tap
+                        ci += BKE;                         // next 128 bytes of channels, or the next tap
                         if (ci >= g.C_in) {
                             ci = 0;
                             if (++kx == g.kw) { kx = 0; ++ky; }
@@ -839,7 +863,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             const int rq = lane >> 3;                      // rows 16pwg + rq + {0,4,8,12}
             // A group owns every second k-block of the whole launch, so its loop steps by two
             // k-blocks: 128 K elements = adv_tap filter taps and adv_ci channels.
-            const int adv_tap = (2 * BK) / g.C_in, adv_ci = (2 * BK) - adv_tap * g.C_in;
+            const int adv_tap = (2 * BKE) / g.C_in, adv_ci = (2 * BKE) - adv_tap * g.C_in;
             // destination of this lane's chunk inside a stage: rows rq, rq + 8 share a swizzle
             // phase, rows rq + 4, rq + 12 the other
             const uint32_t dst_a = (uint32_t)((16 * pwg + rq) * 128 + ((c ^ rq) << 4));
@@ -866,7 +890,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                 // window position (filter tap, channel) of this lane's chunk in k-block kb0
                 int tap, ci;
                 {
-                    const int k_first = kb0 * BK + c * 8;
+                    const int k_first = kb0 * BKE + c * EPC;
                     tap = (int)fd_div((uint32_t)k_first, a.fdCin);
                     ci = k_first - tap * g.C_in;
                 }
@@ -890,7 +914,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                             off = base[i] + rnk * g.C_in + ci;
                         }
                         ptx::cp_async_16(stage + ((i & 1) ? dst_b : dst_a) + (uint32_t)((i >> 1) * 1024),
-                                         x2 + (in ? off : 0), in ? 16u : 0u);
+                                         xb + (in ? (long long)off * ES : 0), in ? 16u : 0u);
                     }
                     ptx::cp_async_mbar_arrive_noinc(ptx::smem_u32(&sh->full[s]));
                     tap += adv_tap;
@@ -1034,10 +1058,12 @@ __global__ void pack_block_filters_kernel(const unsigned short* __restrict__ w, 
 
 }  // namespace
 
-bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fused_list_rows, bool allow_split, FastPlan* plan)
+bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fused_list_rows, bool allow_split, int elem_bytes,
+               FastPlan* plan)
 {
     const int N = g.C_out;
-    const int KB = (g.K + BK - 1) / BK;
+    const int bke = 128 / elem_bytes;             // K elements per stage: 64 bf16 or 32 fp32
+    const int KB = (g.K + bke - 1) / bke;
     const long long m_tiles = (est_kept_rows + BM - 1) / BM > 0 ? (est_kept_rows + BM - 1) / BM : 1;
     // Tile width and k shares.  A wider tile does more work per gathered byte, a narrower one
     // gives more tiles when a layer has few kept rows, and sharing a tile's k-blocks between
@@ -1081,9 +1107,9 @@ bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fuse
     int smem = 1024 + S * stage_bytes + (int)sizeof(Shared) + list_bytes;
     if (smem < 120 * 1024) smem = 120 * 1024;      // one block per SM: tensor memory is not shared out
     plan->smem_bytes = smem;
-    if (g.C_in % 8 != 0) return false;            // the caller pads the channels first
-    plan->vec = (g.C_in % 64 == 0) ? GATHER_TMA : GATHER_CPASYNC;
-    plan->Kpad = ((g.K + BK - 1) / BK) * BK;
+    if (g.C_in % (16 / elem_bytes) != 0) return false;      // the caller pads the channels first
+    plan->vec = (g.C_in % bke == 0) ? GATHER_TMA : GATHER_CPASYNC;
+    plan->Kpad = KB * bke;
     return true;
 }
 
@@ -1091,8 +1117,9 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
                         const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
                         int num_sms, int fuse_compact, long long host_kept, float* ws_partial, int* ws_counters,
-                        int out_compact, const int32_t* in_rank, int in_kept, const void* residual, cudaStream_t st)
+                        int out_compact, const int32_t* in_rank, int in_kept, const void* residual, int f32, cudaStream_t st)
 {
+    if (f32 && (in_rank != nullptr || residual != nullptr || plan.ksplit != 1)) return cudaErrorInvalidValue;
     FastArgs a;
     a.fdcnt_host = make_fastdiv((uint32_t)(host_kept > 0 && host_kept < (1ll << 31) ? host_kept : 1));
     if (!(host_kept > 0 && host_kept < (1ll << 31))) a.fdcnt_host.d = 0;
@@ -1128,7 +1155,7 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     int cols = 32;
     while (cols < 2 * plan.BN) cols <<= 1;
     a.tmem_cols = cols;
-    a.vec_out = (g.C_out % 8 == 0 && (reinterpret_cast<uintptr_t>(y) & 15) == 0) ? 1 : 0;
+    a.vec_out = (g.C_out % (f32 ? 4 : 8) == 0 && (reinterpret_cast<uintptr_t>(y) & 15) == 0) ? 1 : 0;
 
     long long tiles = ((long long)g.M + BM - 1) / BM * plan.n_tiles * plan.ksplit;
     int grid = (int)(tiles < num_sms ? tiles : num_sms);
@@ -1138,15 +1165,19 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     using Kern = void (*)(const CUtensorMap, const CUtensorMap, const ConvGeom, const FastArgs);
     Kern kern = nullptr;
 #define ASX_PICK(MODE, IC)                                                                                          \
-    kern = has_res ? (is_silu ? masked_conv_sm100_kernel<MODE, IC, true, true> : masked_conv_sm100_kernel<MODE, IC, true, false>) \
-                   : (is_silu ? masked_conv_sm100_kernel<MODE, IC, false, true> : masked_conv_sm100_kernel<MODE, IC, false, false>)
-    if (variant == 2) { ASX_PICK(GATHER_TMA, false); }
+    kern = has_res ? (is_silu ? masked_conv_sm100_kernel<MODE, IC, true, true, false> : masked_conv_sm100_kernel<MODE, IC, true, false, false>) \
+                   : (is_silu ? masked_conv_sm100_kernel<MODE, IC, false, true, false> : masked_conv_sm100_kernel<MODE, IC, false, false, false>)
+    if (f32) {      // fp32 storage: dense input, no residual
+        if (variant == 2) kern = is_silu ? masked_conv_sm100_kernel<GATHER_TMA, false, false, true, true> : masked_conv_sm100_kernel<GATHER_TMA, false, false, false, true>;
+        else kern = is_silu ? masked_conv_sm100_kernel<GATHER_CPASYNC, false, false, true, true> : masked_conv_sm100_kernel<GATHER_CPASYNC, false, false, false, true>;
+    }
+    else if (variant == 2) { ASX_PICK(GATHER_TMA, false); }
     else if (variant == 1) { ASX_PICK(GATHER_CPASYNC, false); }
     else if (variant == 4) { ASX_PICK(GATHER_TMA, true); }
     else { ASX_PICK(GATHER_CPASYNC, true); }
 #undef ASX_PICK
-    static int smem_set_all[20] = {0};          // largest dynamic shared memory size enabled so far, per instance
-    int* smem_set = smem_set_all + (has_res ? 5 : 0) + (is_silu ? 10 : 0);
+    static int smem_set_all[40] = {0};          // largest dynamic shared memory size enabled so far, per instance
+    int* smem_set = smem_set_all + (has_res ? 5 : 0) + (is_silu ? 10 : 0) + (f32 ? 20 : 0);
     if (plan.smem_bytes > smem_set[variant]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
         if (e != cudaSuccess) return e;

@@ -10,7 +10,15 @@ namespace asx {
 
 namespace {
 
-__global__ void naive_zero_dropped(ConvGeom g, __nv_bfloat16* __restrict__ y,
+// Element types: bf16 (the default storage) or fp32 (ASX_F32; products of the fp32 values as they
+// are, not of their TF32 parts).
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ void from_f32(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+__device__ __forceinline__ void from_f32(float* p, float v) { *p = v; }
+
+template <typename T>
+__global__ void naive_zero_dropped(ConvGeom g, T* __restrict__ y,
                                    const uint8_t* __restrict__ mask)
 {
     const long long total = (long long)g.M * g.C_out;
@@ -18,13 +26,14 @@ __global__ void naive_zero_dropped(ConvGeom g, __nv_bfloat16* __restrict__ y,
          i += (long long)gridDim.x * blockDim.x) {
         const int row = (int)(i / g.C_out);
         const int p = (g.rows == g.P) ? row % g.P : row;
-        if (mask[p] == 0) y[i] = __ushort_as_bfloat16((unsigned short)0);
+        if (mask[p] == 0) from_f32(y + i, 0.f);
     }
 }
 
-__global__ void naive_kept_rows(ConvGeom g, const __nv_bfloat16* __restrict__ x,
-                                const __nv_bfloat16* __restrict__ w, const float* __restrict__ bias,
-                                __nv_bfloat16* __restrict__ y, const int32_t* __restrict__ kept,
+template <typename T>
+__global__ void naive_kept_rows(ConvGeom g, const T* __restrict__ x,
+                                const T* __restrict__ w, const float* __restrict__ bias,
+                                T* __restrict__ y, const int32_t* __restrict__ kept,
                                 const int32_t* __restrict__ count, int relu)
 {
     const int cnt = *count;
@@ -50,28 +59,34 @@ __global__ void naive_kept_rows(ConvGeom g, const __nv_bfloat16* __restrict__ x,
             for (int kx = 0; kx < g.kw; ++kx) {
                 const int ix = ox * g.stride - g.pad + kx;
                 if (ix < 0 || ix >= g.W) continue;
-                const __nv_bfloat16* xp = x + (((long long)n * g.H + iy) * g.W + ix) * g.C_in;
-                const __nv_bfloat16* wp = w + (((long long)co * g.kh + ky) * g.kw + kx) * g.C_in;
+                const T* xp = x + (((long long)n * g.H + iy) * g.W + ix) * g.C_in;
+                const T* wp = w + (((long long)co * g.kh + ky) * g.kw + kx) * g.C_in;
                 for (int ci = 0; ci < g.C_in; ++ci)
-                    acc = fmaf(__bfloat162float(xp[ci]), __bfloat162float(wp[ci]), acc);
+                    acc = fmaf(to_f32(xp[ci]), to_f32(wp[ci]), acc);
             }
         }
         float v = acc + (bias ? bias[co] : 0.f);
         if (relu == 1) v = fmaxf(v, 0.f);
         if (relu == 2) v = v / (1.f + expf(-v));     // SiLU
-        y[(long long)row * g.C_out + co] = __float2bfloat16_rn(v);
+        from_f32(y + (long long)row * g.C_out + co, v);
     }
 }
 
 }  // namespace
 
 cudaError_t launch_naive(const ConvGeom& g, const void* x, const void* w, const float* bias, void* y,
-                         const uint8_t* mask, const int32_t* kept, const int32_t* count, int relu,
+                         const uint8_t* mask, const int32_t* kept, const int32_t* count, int relu, int f32,
                          cudaStream_t st)
 {
     const long long total = (long long)g.M * g.C_out;
     int blocks = (int)((total + 255) / 256 < 148 * 32 ? (total + 255) / 256 : 148 * 32);
     if (blocks < 1) blocks = 1;
+    if (f32) {
+        naive_zero_dropped<float><<<blocks, 256, 0, st>>>(g, static_cast<float*>(y), mask);
+        naive_kept_rows<float><<<blocks, 256, 0, st>>>(g, static_cast<const float*>(x), static_cast<const float*>(w), bias,
+                                                       static_cast<float*>(y), kept, count, relu);
+        return cudaGetLastError();
+    }
     naive_zero_dropped<<<blocks, 256, 0, st>>>(g, static_cast<__nv_bfloat16*>(y), mask);
     naive_kept_rows<<<blocks, 256, 0, st>>>(g, static_cast<const __nv_bfloat16*>(x),
                                             static_cast<const __nv_bfloat16*>(w), bias,

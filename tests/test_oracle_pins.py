@@ -398,3 +398,24 @@ def test_fp32_storage_equals_library_fp64_conv_on_unrounded_inputs():
     sel = np.array([0, 5, 41, 42, 80])
     np.testing.assert_array_equal(oracle.masked_conv_rows(x, w, b, m, 1, 1, "silu", sel, storage="fp32"),
                                   oracle.masked_conv(x, w, b, m, 1, 1, "silu", storage="fp32").reshape(84, 4)[sel])
+
+
+def test_tf32_operand_keeps_ten_mantissa_bits_and_never_grows():
+    """TF32 has 10 explicit mantissa bits: values with at most 11 significant bits are unchanged,
+    everything else loses less than 2^-10 of its magnitude, towards zero; the result is idempotent."""
+    rng = np.random.default_rng(32)
+    a = np.concatenate([rng.standard_normal(100000).astype(np.float32) * np.float32(10.0) ** rng.integers(-20, 20, 100000).astype(np.float32),
+                        np.array([0.0, -0.0, 1.0, -1.0, 1.0 + 2.0 ** -10, 1.0 + 2.0 ** -11, 3.0 - 2.0 ** -22, np.inf, -np.inf], np.float32)])
+    t = oracle.tf32_operand(a)
+    assert np.array_equal(oracle.tf32_operand(t), t)
+    fin = np.isfinite(a)
+    assert np.all(np.abs(t[fin]) <= np.abs(a[fin])) and np.array_equal(np.signbit(t), np.signbit(a))
+    big = fin & (np.abs(a) > 1e-30)
+    assert np.all(np.abs(a[big].astype(np.float64) - t[big]) < np.abs(a[big].astype(np.float64)) * 2.0 ** -10)
+    assert np.array_equal(t[~fin], a[~fin])
+    # 11 significant bits survive, the twelfth is dropped
+    assert oracle.tf32_operand(np.float32(1.0 + 2.0 ** -10)) == np.float32(1.0 + 2.0 ** -10)
+    assert oracle.tf32_operand(np.float32(1.0 + 2.0 ** -11)) == np.float32(1.0)
+    assert oracle.tf32_operand(np.float32(3.0 - 2.0 ** -22)) == np.float32(3.0 - 2.0 ** -9)
+    ints = np.arange(-2048, 2049, dtype=np.float32)
+    assert np.array_equal(oracle.tf32_operand(ints), ints)

@@ -238,12 +238,14 @@ def make_score(cfg: int, H0: int, W0: int) -> np.ndarray:
     return rng.random((H0, W0), dtype=np.float32)
 
 
-def algorithmic_bytes(spec: LayerSpec, mask: np.ndarray) -> int:
+def algorithmic_bytes(spec: LayerSpec, mask: np.ndarray, elem_bytes: int = 2) -> int:
     """Bytes the method must move for one layer call: touched input pixels, weights,
-    bias, the full output (zero rows included), the mask and the kept-row list."""
+    bias, the full output (zero rows included), the mask and the kept-row list.
+    elem_bytes: storage size of x, w and y (2 for bf16, 4 for fp32)."""
     Pk = int(mask.sum())
     U = touched_input_pixels(spec, mask)
-    return 2 * spec.C_in * U + 2 * spec.K * spec.N + 4 * spec.N + 2 * spec.M * spec.N + mask.size + 4 * Pk
+    e = elem_bytes
+    return e * spec.C_in * U + e * spec.K * spec.N + 4 * spec.N + e * spec.M * spec.N + mask.size + 4 * Pk
 
 
 def iter_small_cases() -> Iterator[LayerSpec]:
