@@ -159,3 +159,37 @@ def test_unsupported_combinations_are_refused():
         rc = layer.run_raw(xd.data_ptr(), spec.Nb, spec.H, spec.W, wd.data_ptr(), 0, out.data_ptr(), asx.F32 | extra, 0)
         assert rc == 2      # ASX_ERR_UNSUPPORTED
     layer.close()
+
+
+def test_resnet18_batch64_stack_full_size_sampled_rows():
+    """Configuration 3 in fp32 storage, launched as `bench.py --dtype f32` launches it (ASX_RECOMPACT,
+    ReLU): kept list and zero rows in full, 768 sampled rows per layer against the oracle."""
+    rng = np.random.default_rng(33)
+    for spec in wl.config(3):
+        x, w, b, mask = tf32_problem(spec)
+        xd, wd, bd = torch.from_numpy(x).cuda(), torch.from_numpy(w).cuda(), torch.from_numpy(b).cuda()
+        y = torch.empty((spec.Nb, spec.Ho, spec.Wo, spec.C_out), dtype=torch.float32, device="cuda")
+        y.view(torch.int32).fill_(0x7fc00001)
+        layer = asx.MaskedConvLayer(spec.C_in, spec.C_out, spec.kh, spec.kw, spec.stride, spec.pad)
+        layer.set_mask(mask)
+        layer.run(xd, wd, bd, out=y, flags=asx.ACT_RELU | asx.RECOMPACT | asx.F32)
+        torch.cuda.synchronize()
+        assert layer.device_status() == 0
+        kept = layer.kept()
+        layer.close()
+        assert np.array_equal(kept, oracle.kept_list(mask)), spec.name
+        y2 = y.view(spec.Nb, spec.P, spec.C_out)
+        md = torch.from_numpy(mask.astype(bool)).cuda()
+        assert not bool(y2[:, ~md, :].view(torch.int32).any()), f"{spec.name}: dropped rows are not all-zero bits"
+        assert not bool(torch.isnan(y2[:, md, :]).any()), f"{spec.name}: a kept element was never written"
+        kept_rows = np.nonzero(np.tile(mask, spec.Nb))[0]
+        sel = rng.choice(kept_rows, size=min(768, kept_rows.size), replace=False)
+        sel = np.unique(np.concatenate([sel, kept_rows[:2], kept_rows[-2:], rng.integers(0, spec.M, 16)])).astype(np.int64)
+        ref = oracle.masked_conv_rows(x, w, b, mask, spec.stride, spec.pad, True, sel, storage="fp32")
+        got = y.view(spec.M, spec.C_out)[torch.from_numpy(sel).cuda()].cpu().numpy().astype(np.float64)
+        diff = got - ref
+        rel = float(np.linalg.norm(diff)) / max(float(np.linalg.norm(ref)), 1e-30)
+        tol = 1e-3 * math.sqrt(spec.K) * float(np.abs(x).max()) * float(np.abs(w).max())
+        assert rel <= REL_TOL_F32, f"{spec.name}: relative Frobenius error {rel:.3e}"
+        assert float(np.abs(diff).max()) <= tol, f"{spec.name}: max abs error {np.abs(diff).max():.3e} > {tol:.3e}"
+        del xd, wd, y, y2
