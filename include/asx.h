@@ -223,16 +223,20 @@ asx_status asx_destroy(asx_layer* layer);
  *   kept_dev  : device, room for `rows` int32; receives the ascending kept positions.
  *   count_dev : device, one int32; receives the number of kept positions.
  *   scratch_dev, scratch_bytes : device scratch of at least asx_compact_scratch_bytes(rows)
- *               bytes, 8-byte aligned; contents on entry are irrelevant, it is cleared on
- *               the stream first.  Calls sharing one scratch buffer must not overlap.
+ *               bytes, 8-byte aligned; contents on entry are irrelevant (every word that is
+ *               read is written first, in stream order).  Calls sharing one scratch buffer
+ *               must not overlap.
+ * Masks of more than 16384 rows take three launches (tile counts, their scan, the ordered
+ * write; the mask is read twice), smaller ones a single block; no block waits for another.
  * 0 <= rows < 2^31.  Asynchronous on `cuda_stream`; allocates nothing.
  */
 int64_t asx_compact_scratch_bytes(int64_t rows);
 asx_status asx_compact(const uint8_t* mask_dev, int64_t rows, int32_t* kept_dev,
                        int32_t* count_dev, void* scratch_dev, int64_t scratch_bytes,
                        void* cuda_stream);
-/* Waits for `cuda_stream`, then reports whether the last asx_compact that used this scratch
- * buffer ran to completion (ASX_OK) or gave up in a bounded wait (ASX_ERR_TIMEOUT). */
+/* Waits for `cuda_stream`, then reports the status word the last asx_compact left in this scratch
+ * buffer: ASX_OK, or ASX_ERR_TIMEOUT if a kernel gave up in a bounded wait (the compaction kernels
+ * have no such wait any more, so this reports ASX_OK after any completed call). */
 asx_status asx_compact_status(const void* scratch_dev, void* cuda_stream);
 
 /*
