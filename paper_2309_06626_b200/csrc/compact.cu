@@ -104,7 +104,7 @@ compact_scan_tiles_kernel(unsigned* __restrict__ tile_count, int num_tiles, int3
         const int i0 = base + tid * PER;
         unsigned v[PER];
 #pragma unroll
-        for (int j = 0; j < PER; ++j) v[j] = i0 + j < num_tiles ? tile_count[i0 + j] : 0u;
+        for (int j = 0; j < PER; ++j) v[j] = i0 + j < num_tiles ? __ldcg(tile_count + i0 + j) : 0u;   // written by the pass before: read past L1
         unsigned mine = 0;
 #pragma unroll
         for (int j = 0; j < PER; ++j) mine += v[j];
@@ -171,7 +171,10 @@ compact_write_kernel(const uint8_t* __restrict__ mask, long long rows, int32_t* 
         if (lane == 31) s_warp_total[sub][warp] = v;
     }
     ptx::grid_dependency_wait();          // the offsets come from the pass before; the list may still be read
-    const int exclusive0 = (int)tile_offset[blockIdx.x];
+    // Read past L1: this block was launched while the passes before were running, L1 is not
+    // invalidated in between, and the SM may hold the line as the counting pass left it (a block of the
+    // first wave runs on the SM where the counting block of the same tile wrote that word).
+    const int exclusive0 = (int)__ldcg(tile_offset + blockIdx.x);
     __syncthreads();
     int base = 0;
 #pragma unroll

@@ -228,10 +228,15 @@ __device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, i
 }
 
 // Output row (n*P + p) of the rk-th kept lowered row.
+// What the kernel before this one in the stream wrote (the list, its count, a residual tensor) is read
+// past L1 (ld.global.cg): a kernel launched as a programmatic dependent starts while its predecessor
+// runs, L1 is not invalidated between the two, and an SM can still hold a line with the older
+// contents of an address (seen with the compaction passes: blocks read the count they had written
+// in the pass before instead of the scanned offset).
 struct KeptList {
     const int32_t* g;            // in global memory, or
     const unsigned short* s;     // this block's 16-bit copy in shared memory (fused compaction)
-    __device__ __forceinline__ int at(int i) const { return s != nullptr ? (int)s[i] : __ldg(g + i); }
+    __device__ __forceinline__ int at(int i) const { return s != nullptr ? (int)s[i] : __ldcg(g + i); }
 };
 __device__ __forceinline__ int out_row_of(int rk, const FastDiv& fdcnt, const ConvGeom& g, const KeptList& kept)
 {
@@ -251,7 +256,7 @@ __device__ __forceinline__ void load_residual8(const __nv_bfloat16* residual, lo
     for (int j = 0; j < 8; ++j) res[j] = 0.f;
     if (residual == nullptr) return;
     if (vec) {
-        const uint4 q = __ldg(reinterpret_cast<const uint4*>(residual + off));
+        const uint4 q = __ldcg(reinterpret_cast<const uint4*>(residual + off));
         const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -261,7 +266,7 @@ __device__ __forceinline__ void load_residual8(const __nv_bfloat16* residual, lo
     } else {
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-            if (j < left) res[j] = __bfloat162float(residual[off + j]);
+            if (j < left) res[j] = __uint_as_float((uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(residual) + off + j) << 16);
     }
 }
 
@@ -405,7 +410,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     // for it here.  With it, the wait comes after the row decoding below, which needs only the list.
     if (!a.fuse_compact) {
         ptx::grid_dependency_wait();
-        cnt = *a.count;
+        cnt = __ldcg(a.count);
     }
     const int Mk = (g.rows == g.P) ? g.Nb * cnt : cnt;
     // With every position dropped there are no tiles; the zero warps then write the whole output

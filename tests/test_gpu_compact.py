@@ -30,6 +30,31 @@ def test_compaction_matches_oracle(rows, q):
     assert np.array_equal(kept, ref)
 
 
+@pytest.mark.parametrize("rows", [16383, 16384, 16385, 16400, 32768, 32769, 16384 * 9 + 4095])
+def test_tile_boundaries_of_the_three_pass_form(rows):
+    """Row counts around the 16384-row tiles of the large-mask passes (one block up to 16384 rows,
+    count / scan / write above), with ragged and exactly full last tiles."""
+    rng = np.random.default_rng(rows)
+    for q in (0.0, 0.37, 1.0):
+        mask = (rng.random(rows) < q).astype(np.uint8)
+        kept, c = _compact(mask)
+        assert np.array_equal(kept, oracle.kept_list(mask))
+
+
+def test_more_tiles_than_one_round_of_the_tile_scan():
+    """2^27 rows and a bit: 8196 tiles, so the one-block scan of the tile counts (8192 per round)
+    carries a running total into a second round; kept runs that straddle tile boundaries."""
+    rows = (1 << 27) + 3 * 16384 + 5
+    rng = np.random.default_rng(27)
+    mask = (rng.random(rows) < 0.5).astype(np.uint8)
+    mask[16384 - 3:16384 + 3] = 1
+    mask[(1 << 27) - 2:(1 << 27) + 2] = 1
+    kept, c = _compact(mask)
+    ref = oracle.kept_list(mask)
+    assert c == ref.size
+    assert np.array_equal(kept, ref)
+
+
 def test_compaction_unaligned_pointer_and_nonbinary_bytes():
     rng = np.random.default_rng(3)
     mask = rng.integers(0, 3, 50001).astype(np.uint8)        # 0, 1 or 2: non-zero keeps
