@@ -37,12 +37,12 @@ L2_BYTES = 126 * 1024 * 1024
 
 # DRAM traffic of the dominant kernel from one ncu capture of the default workload (ResNet-18 stack,
 # batch 64): dram__bytes_read.sum + dram__bytes_write.sum averaged over the 20 fused-kernel launches
-# of a step (12.18 MB read + 2.35 MB written; ncu flushes the caches before every captured launch,
+# of a step (12.18 MB read + 2.37 MB written; ncu flushes the caches before every captured launch,
 # so reads are cold-cache and most of a launch's output is still in L2 when its counters stop).
 # The figure belongs to the kernel sources whose digest is recorded with it; with any other sources
 # the bench reports null.
-NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.52e6,
-               "csrc_sha256": "ba0931ab916cfef771d2806b5f14c20cff627f22dcbbf8bd9199c16c08375c5f"}
+NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.54e6,
+               "csrc_sha256": "fbfd4091dd51ba734e7f9d2fe1af3a30db7a829569e92f869aac216077f4f393"}
 
 
 def csrc_digest() -> str:

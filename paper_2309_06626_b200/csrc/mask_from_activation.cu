@@ -43,7 +43,8 @@ __global__ void __launch_bounds__(256) mask_from_activation_vec_kernel(const uin
     for (long long r0 = warp * rows_per_warp; r0 < rows; r0 += nwarps * rows_per_warp) {
         const long long r = r0 + sub;
         bool p = false;
-        if (r < rows) p = any_positive8(__ldcs(x + r0 * lanes_per_row + lane));     // streamed: read once
+        if (r < rows) p = any_positive8(__ldcg(x + r0 * lanes_per_row + lane));     // read once, and past L1: the
+                                                                                          // kernel before may have written it
         const unsigned b = __ballot_sync(0xffffffffu, p);
         if (r < rows && (lane % lanes_per_row) == 0) mask[r] = (b & group) ? 1 : 0;
     }
@@ -60,7 +61,7 @@ __global__ void __launch_bounds__(256) mask_from_activation_gen_kernel(const uns
     const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
     for (long long r = warp; r < rows; r += nwarps) {
         bool p = false;
-        for (int c = lane; c < C; c += 32) p = p || positive_bf16(x[r * C + c]);
+        for (int c = lane; c < C; c += 32) p = p || positive_bf16(__ldcg(x + r * C + c));
         const unsigned b = __ballot_sync(0xffffffffu, p);
         if (lane == 0) mask[r] = b ? 1 : 0;
     }

@@ -957,7 +957,7 @@ __global__ void pad_channels_kernel(const unsigned short* __restrict__ src, uint
         unsigned short e[8];
 #pragma unroll
         for (int q2 = 0; q2 < 8; ++q2) {
-            e[q2] = (c < C) ? src[row * C + c] : (unsigned short)0;
+            e[q2] = (c < C) ? __ldcg(src + row * C + c) : (unsigned short)0;     // past L1, like everything an earlier kernel may have written
             if (++c == Cp) { c = 0; ++row; }
         }
         uint4 v;
@@ -1013,7 +1013,7 @@ __global__ void stage_blocks2x2_kernel(const unsigned short* __restrict__ x, uin
                 uint32_t q0 = 0, q1 = 0, q2 = 0;
                 if (in) {
                     const uint32_t* src = reinterpret_cast<const uint32_t*>(x + (((long long)n * H + iy) * W + ix) * 3);
-                    q0 = __ldg(src); q1 = __ldg(src + 1); q2 = __ldg(src + 2);
+                    q0 = __ldcg(src); q1 = __ldcg(src + 1); q2 = __ldcg(src + 2);
                 }
                 v[r * 8 + 0] = (unsigned short)(q0 & 0xffffu); v[r * 8 + 1] = (unsigned short)(q0 >> 16);
                 v[r * 8 + 2] = (unsigned short)(q1 & 0xffffu); v[r * 8 + 3] = 0;
@@ -1029,7 +1029,7 @@ __global__ void stage_blocks2x2_kernel(const unsigned short* __restrict__ x, uin
                 const bool in = iy >= 0 && iy < H && ix >= 0 && ix < W;
                 const unsigned short* src = x + (((long long)n * H + (in ? iy : 0)) * W + (in ? ix : 0)) * C;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) v[(r * 2 + px) * 4 + c] = (in && c < C) ? src[c] : (unsigned short)0;
+                for (int c = 0; c < 4; ++c) v[(r * 2 + px) * 4 + c] = (in && c < C) ? __ldcg(src + c) : (unsigned short)0;
             }
         uint4 lo, hi;
         lo.x = v[0] | ((uint32_t)v[1] << 16); lo.y = v[2] | ((uint32_t)v[3] << 16);
