@@ -76,3 +76,20 @@ def test_compaction_repeated_calls_share_scratch():
                                      scratch.data_ptr(), scratch.numel() * 8, st) == 0
     torch.cuda.synchronize()
     assert np.array_equal(kept[:int(count.item())].cpu().numpy(), oracle.kept_list(mask))
+
+
+def test_back_to_back_calls_on_changing_masks():
+    """Several calls in a row, launches overlapping (each pass is a programmatic dependent of the one
+    before), with a different mask, list and scratch every time.  A pass that reads what the pass before
+    wrote through a stale L1 line gets this wrong from the second call on (the first call of a process
+    is serialised by kernel loading and hides it)."""
+    rows = 1 << 24
+    rng = np.random.default_rng(24)
+    masks = [(rng.random(rows) < q).astype(np.uint8) for q in (0.5, 0.2, 0.8, 0.5)]
+    dev = [torch.from_numpy(m).cuda() for m in masks]
+    outs = [asx.compact_mask(d) for d in dev]          # no synchronisation between the calls
+    torch.cuda.synchronize()
+    for m, (kept, count, scratch) in zip(masks, outs):
+        ref = oracle.kept_list(m)
+        assert int(count.item()) == ref.size
+        assert np.array_equal(kept[:ref.size].cpu().numpy(), ref)
