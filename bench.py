@@ -257,9 +257,9 @@ class DeviceLayer:
         self.bytes = wl.algorithmic_bytes(spec, self.mask, 4 if f32 else 2)
         self.ptrs = (self.x.data_ptr(), spec.Nb, spec.H, spec.W, self.w.data_ptr(), self.b.data_ptr(),
                      self.y.data_ptr())
-        # fused kernel (it rebuilds the kept-row list itself for masks of up to 16384 rows, else a
-        # compaction kernel runs first), plus channel padding of x and w when C_in % 8 != 0
-        self.launches = 1 + (0 if self.mask.size <= 16384 else 1) + (2 if spec.C_in % (4 if f32 else 8) else 0)
+        # fused kernel (it rebuilds the kept-row list itself for masks of up to 16384 rows, else the three
+        # compaction passes run first), plus channel padding of x and w when C_in % 8 != 0
+        self.launches = 1 + (0 if self.mask.size <= 16384 else 3) + (2 if spec.C_in % (4 if f32 else 8) else 0)
 
     def step(self, st, flags, layer=None):
         L = layer or self.layer
