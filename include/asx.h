@@ -58,8 +58,13 @@ enum {
     ASX_IN_COMPACT = 16,   /* x holds only the positions kept by the mask given to asx_set_input_mask */
     ASX_ACT_SILU = 32,     /* y = z / (1 + exp(-z)), z = acc + bias, on kept rows (the activation of the YOLOv5
                               network of Section 4); not together with ASX_ACT_RELU (ASX_ERR_INVALID_ARG) */
-    ASX_F32 = 64           /* x, w and y are fp32, the storage type of Appendix A, Algorithm 2 (its sizeof(float));
+    ASX_F32 = 64,          /* x, w and y are fp32, the storage type of Appendix A, Algorithm 2 (its sizeof(float));
                               the products run on the tensor cores in TF32, see asx_run */
+    ASX_IMPL_ROW_GATHER = 128  /* always build the lowered rows by gathering every filter tap of every kept row
+                              separately (the general form of the producer), also where the library would load a
+                              tile's window range once and cut the taps out of it (stride-1 layers with several
+                              taps and C_in % 64 == 0 whose mask came from host memory).  Same results up to
+                              summation order; a tuning and test switch */
 };
 
 /* Human-readable name of a status code; never NULL; static storage. */
@@ -165,7 +170,8 @@ asx_status asx_recompact(asx_layer* layer, void* cuda_stream);
  *   bias : device, fp32 [C_out], 4-byte aligned, or NULL for zero bias.
  *   y    : device, bf16 [Nb][Ho][Wo][C_out], Ho = (H + 2*pad - kh)/stride + 1 (Wo alike);
  *          16-byte aligned when C_out % 8 == 0, else 2-byte; must not overlap x.
- *   flags: OR of ASX_ACT_RELU or ASX_ACT_SILU, ASX_RECOMPACT, ASX_IMPL_NAIVE, ASX_OUT_COMPACT, ASX_IN_COMPACT, ASX_F32.
+ *   flags: OR of ASX_ACT_RELU or ASX_ACT_SILU, ASX_RECOMPACT, ASX_IMPL_NAIVE, ASX_OUT_COMPACT, ASX_IN_COMPACT, ASX_F32,
+ *          ASX_IMPL_ROW_GATHER.
  *          Dropped positions are 0 under every activation (each maps 0 to 0; no bias is added there).  With
  *          ASX_OUT_COMPACT y is bf16 [Nb*P'][C_out] (P' = kept entries of the mask, which must then be
  *          shared by the batch); with ASX_IN_COMPACT x is bf16 [Nb*P'_in][C_in] (see asx_set_input_mask).
@@ -213,6 +219,25 @@ asx_status asx_get_mask(asx_layer* layer, uint8_t* host_mask_out, int64_t rows);
  * call is then undefined; the CUDA context stays usable).  The word is cleared by the call.
  */
 asx_status asx_last_device_status(asx_layer* layer);
+
+/*
+ * Which form of the lowering (Section 3.2, stage i) the last asx_run on this layer used:
+ *   ASX_FORM_NONE (no run yet), ASX_FORM_NAIVE (ASX_IMPL_NAIVE), ASX_FORM_ROW_GATHER_COPY (16-byte copies per
+ *   filter tap and kept row), ASX_FORM_ROW_GATHER_TMA (TMA row gather per filter tap and kept row),
+ *   ASX_FORM_WINDOW_PATCH (a tile's window range loaded once, filter taps cut out of it into tensor memory).
+ * All forms compute the same result up to summation order; this only reports the choice (tests, tuning).
+ */
+enum { ASX_FORM_NONE = 0, ASX_FORM_NAIVE = 1, ASX_FORM_ROW_GATHER_COPY = 2, ASX_FORM_ROW_GATHER_TMA = 3, ASX_FORM_WINDOW_PATCH = 4 };
+asx_status asx_last_run_form(const asx_layer* layer, int* form);
+
+/*
+ * Bound of every wait inside the fused kernels of this layer (on a pipeline barrier or on another
+ * block's partial sums), in GPU clock cycles; cycles <= 0 restores the default of about two seconds.
+ * A wait that runs out makes every role of the kernel leave, the call's output is undefined and
+ * asx_last_device_status reports ASX_ERR_TIMEOUT; the next asx_run starts clean.  The method itself has
+ * no such notion (the paper runs on one CPU thread pool); this is a property of the GPU pipeline.
+ */
+asx_status asx_set_wait_limit(asx_layer* layer, int64_t cycles);
 
 /* Free the layer and the device memory it owns.  NULL is allowed. */
 asx_status asx_destroy(asx_layer* layer);

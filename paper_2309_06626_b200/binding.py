@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libasx.so")
 _lib = None
 
-ACT_RELU, RECOMPACT, IMPL_NAIVE, OUT_COMPACT, IN_COMPACT, ACT_SILU, F32 = 1, 2, 4, 8, 16, 32, 64
+ACT_RELU, RECOMPACT, IMPL_NAIVE, OUT_COMPACT, IN_COMPACT, ACT_SILU, F32, IMPL_ROW_GATHER = 1, 2, 4, 8, 16, 32, 64, 128
 
 # every symbol include/asx.h declares
 EXPORTS = (
@@ -17,8 +17,10 @@ EXPORTS = (
     "asx_get_kept", "asx_get_kept_host", "asx_get_mask", "asx_last_device_status", "asx_destroy",
     "asx_compact_scratch_bytes", "asx_compact", "asx_compact_status", "asx_compact_static",
     "asx_mask_from_scores", "asx_set_mask_from_scores", "asx_mask_from_activation", "asx_set_input_mask", "asx_set_residual",
+    "asx_last_run_form", "asx_set_wait_limit",
 )
 COMPACT_STATIC_MAX_ROWS = 1 << 24
+FORM_NONE, FORM_NAIVE, FORM_ROW_GATHER_COPY, FORM_ROW_GATHER_TMA, FORM_WINDOW_PATCH = 0, 1, 2, 3, 4
 
 
 class AsxError(RuntimeError):
@@ -60,6 +62,8 @@ def lib():
         L.asx_compact_static.argtypes = [vp, i64, vp, vp, vp]
         L.asx_set_input_mask.argtypes = [vp, vp, i64, vp]
         L.asx_set_residual.argtypes = [vp, vp]
+        L.asx_last_run_form.argtypes = [vp, ctypes.POINTER(ci)]
+        L.asx_set_wait_limit.argtypes = [vp, i64]
         L.asx_mask_from_activation.argtypes = [vp, i64, ci, vp, vp]
         L.asx_mask_from_scores.argtypes = [vp, ci, ci, ci, ci, ctypes.c_double, vp]
         L.asx_set_mask_from_scores.argtypes = [vp, vp, ci, ci, ci, ci, ctypes.c_double, vp]
@@ -137,6 +141,15 @@ class MaskedConvLayer:
         sc = np.ascontiguousarray(score, dtype=np.float32)
         _check(lib().asx_set_mask_from_scores(self._h, sc.ctypes.data, sc.shape[0], sc.shape[1], Ho, Wo,
                                               float(sparsity), _stream_ptr(stream)), "asx_set_mask_from_scores")
+
+    def last_run_form(self) -> int:
+        """Producer form of the last run (the FORM_* constants)."""
+        f = ctypes.c_int(0)
+        _check(lib().asx_last_run_form(self._h, ctypes.byref(f)), "asx_last_run_form")
+        return f.value
+
+    def set_wait_limit(self, cycles: int) -> None:
+        _check(lib().asx_set_wait_limit(self._h, int(cycles)), "asx_set_wait_limit")
 
     def recompact(self, stream=None) -> None:
         _check(lib().asx_recompact(self._h, _stream_ptr(stream)), "asx_recompact")

@@ -47,6 +47,22 @@ struct asx_layer {
     int64_t tmapx_pixels = 0;
     int tmapx_stride = 0;              // bytes between rows of the input view
     cudaStream_t last_stream = nullptr;
+    // what the host knows about the current mask (masks that came from host memory, up to 2^24 rows)
+    std::vector<uint8_t> host_mask;
+    uint64_t mask_epoch = 0;           // bumped by every asx_set_mask*
+    // window-patch form: rows of padded input the windows of one 128-row tile span at most, cached per geometry
+    // window-patch form: the row tiles cut from the host's mask, cached per geometry and buffer size
+    uint64_t tiles_epoch = ~0ull;
+    int tiles_Nb = 0, tiles_H = 0, tiles_W = 0, tiles_cap = 0;
+    std::vector<int32_t> host_tiles;   // pairs: first kept lowered row, rows
+    int64_t tiles_rows = 0;            // kept lowered rows they cover
+    void* d_tiles = nullptr;
+    size_t d_tiles_bytes = 0;
+    CUtensorMap tmap_x4;               // x as a 4-D tensor (C_in, W, H, Nb) with one padded row of 64 channels per box
+    const void* tmapx4_ptr = nullptr;
+    int tmapx4_Nb = 0, tmapx4_H = 0, tmapx4_W = 0, tmapx4_Wp = 0;
+    int wait_limit_kcycles = 0;
+    int last_form = ASX_FORM_NONE;     // producer form of the last asx_run        // bound of the in-kernel waits in units of 1024 cycles (0: the default, about 2 s)
 };
 
 namespace {
@@ -134,6 +150,39 @@ void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
+// Window-patch form: cut the kept lowered rows (ascending in image and output row) into tiles of at
+// most 128 consecutive rows whose windows span at most `cap` zero-padded input rows.  Pure index
+// bookkeeping on the mask the host holds; returns the kept lowered rows, or -1 without memory.
+int64_t cut_row_tiles(const std::vector<uint8_t>& mask, int Nb, int P, int Wo, int Hp, int kh, int cap, std::vector<int32_t>* tiles)
+{
+    std::vector<int32_t> kept;
+    tiles->clear();
+    try {
+        kept.reserve(mask.size());
+        for (size_t i = 0; i < mask.size(); ++i)
+            if (mask[i] != 0) kept.push_back((int32_t)i);
+        const bool shared = (int64_t)mask.size() == (int64_t)P;
+        const int64_t Pk = (int64_t)kept.size(), Mk = shared ? Pk * Nb : Pk;
+        auto padded_row = [&](int64_t rk) -> int64_t {
+            const int64_t row = shared ? (rk / Pk) * P + kept[(size_t)(rk % Pk)] : kept[(size_t)rk];
+            return (row / P) * Hp + (row % P) / Wo;
+        };
+        tiles->reserve((size_t)(Mk / 64 + 2));
+        for (int64_t r0 = 0; r0 < Mk;) {
+            const int64_t first = padded_row(r0);
+            int64_t n = 1;
+            while (n < 128 && r0 + n < Mk && padded_row(r0 + n) - first + kh <= cap) ++n;
+            tiles->push_back((int32_t)r0);
+            tiles->push_back((int32_t)n);
+            r0 += n;
+        }
+        return Mk;
+    } catch (const std::bad_alloc&) {
+        tiles->clear();
+        return -1;
+    }
+}
+
 }  // namespace
 
 extern "C" {
@@ -187,16 +236,26 @@ asx_status asx_set_mask(asx_layer* L, const uint8_t* mask, int64_t rows, void* c
     if (on_device) {
         e = cudaMemcpyAsync(L->d_mask, mask, (size_t)rows, cudaMemcpyDeviceToDevice, st);
         L->host_kept = -1;
+        L->host_mask.clear();
     } else {
         int64_t kept = 0;                                         // only sizes the tiles (a launch heuristic)
         for (int64_t i = 0; i < rows; ++i) kept += mask[i] != 0;
         L->host_kept = kept;
+        L->host_mask.clear();
+        if (rows <= (1ll << 24)) {
+            try {
+                L->host_mask.assign(mask, mask + rows);
+            } catch (const std::bad_alloc&) {
+                L->host_mask.clear();                              // only costs the choice of kernel form
+            }
+        }
         e = cudaMemcpyAsync(L->d_mask, mask, (size_t)rows, cudaMemcpyHostToDevice, st);
         if (e == cudaSuccess) e = cudaStreamSynchronize(st);      // the caller may free a host mask on return
     }
     if (e != cudaSuccess) return from_cuda(e);
     L->rows = rows;
     L->last_stream = st;
+    ++L->mask_epoch;
     s = run_compaction(L, st);
     L->has_mask = (s == ASX_OK);
     return s;
@@ -348,7 +407,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
 {
     if (L == nullptr || x == nullptr || w == nullptr || y == nullptr) return ASX_ERR_INVALID_ARG;
     if (Nb < 1 || H < 1 || W < 1) return ASX_ERR_INVALID_ARG;
-    if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE | ASX_OUT_COMPACT | ASX_IN_COMPACT | ASX_ACT_SILU | ASX_F32)) return ASX_ERR_INVALID_ARG;
+    if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE | ASX_OUT_COMPACT | ASX_IN_COMPACT | ASX_ACT_SILU | ASX_F32 | ASX_IMPL_ROW_GATHER)) return ASX_ERR_INVALID_ARG;
     const bool f32 = (flags & ASX_F32) != 0;
     const int ES = f32 ? 4 : 2;                 // bytes per element of x, w and y
     const int EPC = 16 / ES;                    // elements per 16-byte chunk
@@ -412,6 +471,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     int32_t* d_count = L->d_small;
     int* d_status = reinterpret_cast<int*>(L->d_small + 1);
 
+    if (flags & ASX_IMPL_NAIVE) L->last_form = ASX_FORM_NAIVE;
     if (flags & ASX_IMPL_NAIVE)
         return from_cuda(launch_naive(g, x, w, bias, y, L->d_mask, L->d_kept, d_count, relu, f32 ? 1 : 0, st));
 
@@ -556,7 +616,36 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     // and 16-byte output stores.
     const bool allow_split = !f32 && L->host_kept >= 0 && L->C_out % 8 == 0 && (reinterpret_cast<uintptr_t>(y) & 15) == 0;
     if (!plan_fast(g, L->num_sms, est_rows, fuse_compact ? (int)L->rows : 0, allow_split, ES, &plan)) return ASX_ERR_UNSUPPORTED;
-    if (plan.ksplit > 1) {
+    // Stride-1 layers with several filter taps and whole 64-channel slices take the window-patch form
+    // when the host knows the mask, every tile's windows fit the patch buffers and the planner's
+    // estimate favours it; compact tensors and fp32 storage stay with the row gather.
+    PatchPlan pplan;
+    bool use_patch = false;
+    if (!f32 && !in_compact && !out_compact && !(flags & ASX_IMPL_ROW_GATHER) && !L->host_mask.empty() &&
+        (reinterpret_cast<uintptr_t>(y) & 15) == 0 && plan_patch(g, fuse_compact ? (int)L->rows : 0, &pplan)) {
+        if (L->tiles_epoch != L->mask_epoch || L->tiles_Nb != Nb || L->tiles_H != H || L->tiles_W != W || L->tiles_cap != pplan.cap_rows) {
+            L->tiles_rows = cut_row_tiles(L->host_mask, Nb, g.P, g.Wo, pplan.Hp, g.kh, pplan.cap_rows, &L->host_tiles);
+            L->tiles_epoch = L->mask_epoch; L->tiles_Nb = Nb; L->tiles_H = H; L->tiles_W = W; L->tiles_cap = pplan.cap_rows;
+            const size_t need = L->host_tiles.size() * sizeof(int32_t);
+            if (L->tiles_rows > 0 && need > 0) {
+                if (need > L->d_tiles_bytes) {
+                    cudaStreamSynchronize(st);
+                    cudaFree(L->d_tiles);
+                    L->d_tiles = nullptr; L->d_tiles_bytes = 0;
+                    if (cudaMalloc(&L->d_tiles, need) != cudaSuccess) return ASX_ERR_OOM;
+                    L->d_tiles_bytes = need;
+                }
+                // ordered on the stream behind any launch that still reads the old table; host_tiles lives on in the layer
+                if (cudaMemcpyAsync(L->d_tiles, L->host_tiles.data(), need, cudaMemcpyHostToDevice, st) != cudaSuccess) return ASX_ERR_CUDA;
+                if (cudaStreamSynchronize(st) != cudaSuccess) return ASX_ERR_CUDA;
+            }
+        }
+        if (L->tiles_rows > 0 && L->tiles_rows == est_rows) {
+            plan_patch_cost(g, L->num_sms, (long long)(L->host_tiles.size() / 2), &pplan);
+            use_patch = pplan.est_cost_us <= plan.est_cost_us;
+        }
+    }
+    if (plan.ksplit > 1 && !use_patch) {
         const size_t need = (size_t)plan.ws_items * 128 * (size_t)plan.BN * sizeof(float);
         if (need > L->ws_bytes) {
             cudaFree(L->d_ws);
@@ -573,21 +662,41 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
             if (cudaMemsetAsync(L->d_wscnt, 0, ints * sizeof(int), st) != cudaSuccess) return ASX_ERR_CUDA;
         }
     }
+    const int BNsel = use_patch ? pplan.BN : plan.BN;
     const int Kw = g.K;
     const CUtensorMapDataType tm_type = f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     const cuuint32_t box_k = (cuuint32_t)(128 / ES);           // one 128-byte swizzled row of K elements
-    if (L->tmap_ptr != wsrc || L->tmap_BN != plan.BN || L->tmap_Kw != Kw || L->tmap_es != ES) {
+    if (L->tmap_ptr != wsrc || L->tmap_BN != BNsel || L->tmap_Kw != Kw || L->tmap_es != ES) {
         EncodeTiledFn enc = encode_tiled_fn();
         if (enc == nullptr) return ASX_ERR_CUDA;
         const cuuint64_t dims[2] = {(cuuint64_t)Kw, (cuuint64_t)L->C_out};
         const cuuint64_t strides[1] = {(cuuint64_t)Kw * ES};
-        const cuuint32_t box[2] = {box_k, (cuuint32_t)plan.BN};
+        const cuuint32_t box[2] = {box_k, (cuuint32_t)BNsel};
         const cuuint32_t estr[2] = {1u, 1u};
         const CUresult r = enc(&L->tmap, tm_type, 2, const_cast<void*>(wsrc), dims,
                                strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return ASX_ERR_CUDA;
-        L->tmap_ptr = wsrc; L->tmap_BN = plan.BN; L->tmap_Kw = Kw; L->tmap_es = ES;
+        L->tmap_ptr = wsrc; L->tmap_BN = BNsel; L->tmap_Kw = Kw; L->tmap_es = ES;
+    }
+    if (use_patch) {
+        if (L->tmapx4_ptr != xsrc || L->tmapx4_Nb != Nb || L->tmapx4_H != g.H || L->tmapx4_W != g.W || L->tmapx4_Wp != pplan.Wp) {
+            EncodeTiledFn enc = encode_tiled_fn();
+            if (enc == nullptr) return ASX_ERR_CUDA;
+            const cuuint64_t dims[4] = {(cuuint64_t)g.C_in, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)Nb};
+            const cuuint64_t strides[3] = {(cuuint64_t)g.C_in * 2, (cuuint64_t)g.W * g.C_in * 2, (cuuint64_t)g.H * g.W * g.C_in * 2};
+            const cuuint32_t box[4] = {64u, (cuuint32_t)pplan.Wp, 1u, 1u};
+            const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+            const CUresult r = enc(&L->tmap_x4, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(xsrc), dims, strides, box, estr,
+                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) return ASX_ERR_CUDA;
+            L->tmapx4_ptr = xsrc; L->tmapx4_Nb = Nb; L->tmapx4_H = g.H; L->tmapx4_W = g.W; L->tmapx4_Wp = pplan.Wp;
+        }
+        L->last_form = ASX_FORM_WINDOW_PATCH;
+        return from_cuda(launch_patch(g, pplan, L->tmap, L->tmap_x4, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status, L->num_sms,
+                                      fuse_compact ? 1 : 0, L->host_kept, L->residual, L->d_tiles, (int)(L->host_tiles.size() / 2), L->tiles_rows,
+                                      L->wait_limit_kcycles, st));
     }
     if (plan.vec == 2) {
         const int64_t pixels = in_compact ? x_rows : (int64_t)Nb * g.H * g.W;
@@ -606,9 +715,10 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
             L->tmapx_ptr = xsrc; L->tmapx_pixels = pixels; L->tmapx_stride = row_stride; L->tmapx_es = ES;
         }
     }
+    L->last_form = plan.vec == 2 ? ASX_FORM_ROW_GATHER_TMA : ASX_FORM_ROW_GATHER_COPY;
     return from_cuda(launch_fast(g, plan, L->tmap, plan.vec == 2 ? L->tmap_x : L->tmap, xsrc, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status,
                                  L->num_sms, fuse_compact ? 1 : 0, L->host_kept, static_cast<float*>(L->d_ws), L->d_wscnt,
-                                 out_compact ? 1 : 0, in_compact ? L->d_in_rank : nullptr, (int)L->in_kept, L->residual, f32 ? 1 : 0, st));
+                                 out_compact ? 1 : 0, in_compact ? L->d_in_rank : nullptr, (int)L->in_kept, L->residual, f32 ? 1 : 0, L->wait_limit_kcycles, st));
 }
 
 asx_status asx_get_kept(asx_layer* L, int64_t* count, const int32_t** dev_kept)
@@ -663,13 +773,32 @@ asx_status asx_last_device_status(asx_layer* L)
     return (word != 0 || scan_err != 0) ? ASX_ERR_TIMEOUT : ASX_OK;
 }
 
+asx_status asx_last_run_form(const asx_layer* L, int* form)
+{
+    if (L == nullptr || form == nullptr) return ASX_ERR_INVALID_ARG;
+    *form = L->last_form;
+    return ASX_OK;
+}
+
+asx_status asx_set_wait_limit(asx_layer* L, int64_t cycles)
+{
+    if (L == nullptr) return ASX_ERR_INVALID_ARG;
+    if (cycles <= 0) {
+        L->wait_limit_kcycles = 0;
+    } else {
+        const int64_t k = (cycles + 1023) / 1024;
+        L->wait_limit_kcycles = (int)std::min<int64_t>(k, 1 << 30);
+    }
+    return ASX_OK;
+}
+
 asx_status asx_destroy(asx_layer* L)
 {
     if (L == nullptr) return ASX_OK;
     if (L->device >= 0) {
         cudaStreamSynchronize(L->last_stream);
         cudaFree(L->d_mask); cudaFree(L->d_kept); cudaFree(L->d_scratch);
-        cudaFree(L->d_small); cudaFree(L->d_wpack); cudaFree(L->d_xpad); cudaFree(L->d_ws); cudaFree(L->d_wscnt); cudaFree(L->d_in_rank);
+        cudaFree(L->d_small); cudaFree(L->d_wpack); cudaFree(L->d_xpad); cudaFree(L->d_ws); cudaFree(L->d_wscnt); cudaFree(L->d_in_rank); cudaFree(L->d_tiles);
     }
     delete L;
     return ASX_OK;

@@ -19,7 +19,7 @@ struct ConvGeom {
 };
 
 // Device status word values (bit flags), reported as ASX_ERR_TIMEOUT.
-enum : int { DEV_OK = 0, DEV_TIMEOUT_SCAN = 1, DEV_TIMEOUT_PIPE = 2, DEV_BAD_INDEX = 4 };
+enum : int { DEV_OK = 0, DEV_TIMEOUT_PIPE = 2, DEV_BAD_INDEX = 4 };
 
 // Launch with the programmatic-stream-serialization attribute: the kernel may begin while its
 // predecessor in the stream is still running and must execute griddepcontrol.wait before it
@@ -63,9 +63,9 @@ struct FastPlan {
     int smem_bytes;
     int vec;          // gather mode: 1 cp.async 16 B (a pixel's channels are whole 16-byte chunks), 2 TMA row
                       // gather (they are whole 128-byte runs)
-    int Kpad;         // K rounded up to a whole number of stages
     int ksplit;       // work items per output tile (shares of the k-blocks); > 1 needs the workspace
     long long ws_items;   // m_tiles * n_tiles * ksplit for the estimated kept rows
+    double est_cost_us;   // the planner's estimate of the launch's duration
 };
 // elem_bytes: 2 (bf16 storage) or 4 (fp32 storage, TF32 contraction)
 bool plan_fast(const ConvGeom& g, int num_sms, long long est_kept_rows, int fused_list_rows, bool allow_split, int elem_bytes,
@@ -74,7 +74,29 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
                         const CUtensorMap& tmap_x, const void* x, const float* bias, void* y, const uint8_t* mask,
                         const int32_t* kept, const int32_t* count, int relu, int* dev_status,
                         int num_sms, int fuse_compact, long long host_kept, float* ws_partial, int* ws_counters,
-                        int out_compact, const int32_t* in_rank, int in_kept, const void* residual, int f32, cudaStream_t st);
+                        int out_compact, const int32_t* in_rank, int in_kept, const void* residual, int f32, int wait_limit_kcycles,
+                        cudaStream_t st);
+// ---- the window-patch form of the tensor-core path (masked_conv_patch_sm100.cu): stride-1 layers with
+// several filter taps and C_in % 64 == 0, bf16, dense input and output
+struct PatchPlan {
+    int BN, n_tiles;
+    int a_stages, b_stages;
+    int G;                 // filter taps per pipeline stage
+    int cap_rows;          // padded input rows one patch buffer holds: every tile's windows must span at most this many
+    int Hp, Wp, Wp8;       // padded input height and width, Wp rounded up to a multiple of 8
+    int smem_bytes;
+    double est_cost_us;    // the planner's estimate of the launch's duration
+};
+// false: this geometry does not take the window-patch form
+bool plan_patch(const ConvGeom& g, int fused_list_rows, PatchPlan* plan);
+// fills plan->est_cost_us for a mask that the host cut into n_mtiles row tiles
+void plan_patch_cost(const ConvGeom& g, int num_sms, long long n_mtiles, PatchPlan* plan);
+// tmap_x4: x as a 4-D tensor (C_in, W, H, Nb) with box (64, Wp, 1, 1), 128-byte swizzle, zero fill
+cudaError_t launch_patch(const ConvGeom& g, const PatchPlan& plan, const CUtensorMap& tmap_w, const CUtensorMap& tmap_x4,
+                         const float* bias, void* y, const uint8_t* mask, const int32_t* kept, const int32_t* count,
+                         int relu, int* dev_status, int num_sms, int fuse_compact, long long host_kept,
+                         const void* residual, const void* tiles, int n_mtiles, long long kept_rows, int wait_limit_kcycles,
+                         cudaStream_t st);
 // src[rows][C] -> dst[rows][Cp] with zero channels added (Cp = 4 or a multiple of 8; rows*Cp % 8 == 0)
 cudaError_t launch_pad_channels(const void* src, void* dst, long long rows, int C, int Cp, cudaStream_t st);
 // filters for the pixel-pair form: w[C_out][kh][kw][C] -> w2[C_out][kh][kw2][2][4], where pair kxx,

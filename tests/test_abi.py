@@ -60,7 +60,7 @@ def test_create_layer_argument_checks(L):
     assert L.asx_run(h, None, 1, 8, 8, None, None, None, 0, None) == 1
     buf = (ctypes.c_char * 64)()
     p = ctypes.addressof(buf)
-    assert L.asx_run(h, p, 1, 8, 8, p, None, p, 128, None) == 1      # unknown flag
+    assert L.asx_run(h, p, 1, 8, 8, p, None, p, 1 << 20, None) == 1  # unknown flag
     assert L.asx_run(h, p, 1, 8, 8, p, None, p, 64 | 8, None) == 2   # fp32 storage with a compact output: unsupported
     assert L.asx_run(h, p, 1, 8, 8, p, None, p, 0, None) == 3        # no mask yet
     assert L.asx_get_kept(h, None, None) == 3

@@ -17,7 +17,7 @@ from philox_ref import random_block_mask
 pytestmark = pytest.mark.gpu
 
 SMALL = list(wl.iter_small_cases())
-IMPLS = [("naive", asx.IMPL_NAIVE), ("tcgen05", 0)]
+IMPLS = [("naive", asx.IMPL_NAIVE), ("tcgen05", 0), ("row_gather", asx.IMPL_ROW_GATHER)]
 
 
 @pytest.mark.parametrize("impl", IMPLS, ids=[i[0] for i in IMPLS])

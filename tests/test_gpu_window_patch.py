@@ -1,0 +1,178 @@
+"""The window-patch form of the fused kernel (a tile's window range loaded once into shared memory, the
+filter taps cut out of it into tensor memory) against the CPU oracle, and against the row-gather form.
+
+The library takes this form by itself for stride-1 layers with several filter taps and C_in % 64 == 0
+whose mask came from host memory and whose tiles' windows fit the patch buffers; every case below
+asserts which form ran, so that a silent change of the choice cannot turn these into tests of the
+other form."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2309_06626_b200 as asx
+import workloads as wl
+from gpu_util import check_against_oracle, make_problem, max_abs_tol, to_dev_bf16, REL_FROB_TOL
+
+pytestmark = pytest.mark.gpu
+
+
+def run_form(spec, x, w, b, mask, flags):
+    """Runs the layer and returns (y float64 [M][N], bits, form)."""
+    layer = asx.MaskedConvLayer(spec.C_in, spec.C_out, spec.kh, spec.kw, spec.stride, spec.pad)
+    layer.set_mask(mask)
+    xd, wd = to_dev_bf16(x), to_dev_bf16(w)
+    bd = None if b is None else torch.from_numpy(b).cuda()
+    out = torch.empty((spec.Nb, spec.Ho, spec.Wo, spec.C_out), dtype=torch.bfloat16, device="cuda")
+    out.view(torch.int16).fill_(0x7fc1)
+    layer.run(xd, wd, bd, out=out, flags=flags)
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0
+    form = layer.last_run_form()
+    layer.close()
+    bits = out.view(torch.int16).cpu().numpy().view(np.uint16).reshape(spec.M, spec.C_out)
+    return out.float().cpu().numpy().astype(np.float64).reshape(spec.M, spec.C_out), bits, form
+
+
+def spec_of(name, cin, cout, kh, kw, pad, H, W, Nb, pct, blk, seed):
+    return wl.LayerSpec(name, cin, cout, kh, kw, 1, pad, H, W, Nb, pct, blk, "relu", wl.BASE_SEED + 7000 + seed)
+
+
+CASES = [
+    # name, C_in, C_out, kh, kw, pad, H, W, Nb, pct, block
+    ("p_3x3_c64_n64", 64, 64, 3, 3, 1, 20, 23, 2, 30, 1),
+    ("p_3x3_c64_n64_dense", 64, 64, 3, 3, 1, 20, 23, 2, 0, 1),
+    ("p_3x3_c64_56", 64, 64, 3, 3, 1, 56, 56, 3, 50, 4),          # the ResNet layer1 shape
+    ("p_3x3_c128_28", 128, 128, 3, 3, 1, 28, 28, 4, 50, 4),       # layer2: two slices
+    ("p_3x3_c256_14", 256, 256, 3, 3, 1, 14, 14, 6, 50, 4),       # layer3: tiles cross image borders, two column tiles
+    ("p_3x3_c64_n24", 64, 24, 3, 3, 1, 17, 19, 2, 25, 1),         # narrow tile (BN = 32), odd width
+    ("p_3x3_c64_n200", 64, 200, 3, 3, 1, 12, 13, 2, 40, 2),       # two column tiles of 112, the second ragged
+    ("p_5x5_c64", 64, 40, 5, 5, 2, 15, 13, 2, 50, 1),
+    ("p_2x2_c64_p0", 64, 32, 2, 2, 0, 16, 16, 3, 50, 1),
+    ("p_1x3_c64", 64, 32, 1, 3, 1, 9, 30, 2, 30, 1),              # pad applies to both axes: Ho = H + 2
+    ("p_3x1_c64_p0", 64, 32, 3, 1, 0, 12, 10, 2, 30, 1),
+    ("p_3x3_c320", 320, 72, 3, 3, 1, 12, 12, 1, 10, 1),           # five slices
+    ("p_3x3_c64_p2", 64, 64, 3, 3, 2, 10, 11, 2, 20, 1),          # padding wider than the filter needs
+    ("p_7x7_c64", 64, 16, 7, 7, 3, 12, 12, 2, 50, 2),
+]
+
+
+@pytest.mark.parametrize("case", CASES, ids=[c[0] for c in CASES])
+@pytest.mark.parametrize("act", [asx.ACT_RELU, 0, asx.ACT_SILU], ids=["relu", "none", "silu"])
+def test_window_patch_against_oracle(case, act):
+    spec = spec_of(*case, seed=CASES.index(case))
+    x, w, b, mask = make_problem(spec)
+    layer = asx.MaskedConvLayer(spec.C_in, spec.C_out, spec.kh, spec.kw, 1, spec.pad)
+    layer.set_mask(mask)
+    layer.run(to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda(), flags=act)
+    torch.cuda.synchronize()
+    assert layer.last_run_form() == asx.FORM_WINDOW_PATCH, "this case is meant to take the window-patch form"
+    layer.close()
+    check_against_oracle(spec, x, w, b, mask, act)
+    check_against_oracle(spec, x, w, b, mask, act | asx.RECOMPACT)
+
+
+@pytest.mark.parametrize("kept_rows", [0, 1, 127, 128, 129, 255, 256, 257, "all"])
+def test_tile_boundaries(kept_rows):
+    spec = wl.LayerSpec("edge64", 64, 32, 3, 3, 1, 1, 20, 20, 1, 0, 1, "relu", 4243)
+    x, w, b, _ = make_problem(spec)
+    mask = np.zeros(spec.P, np.uint8)
+    if kept_rows == "all":
+        mask[:] = 1
+    else:
+        mask[np.random.default_rng(kept_rows).permutation(spec.P)[:kept_rows]] = 1
+    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU)
+    y, bits, form = run_form(spec, x, w, b, mask, asx.ACT_RELU)
+    assert form == asx.FORM_WINDOW_PATCH or kept_rows == 0      # with nothing kept there are no tiles to cut
+
+
+def test_per_row_mask():
+    spec = spec_of("p_rowmask", 64, 64, 3, 3, 1, 18, 21, 3, 40, 2, seed=50)
+    x, w, b, mask = make_problem(spec, per_row=True)
+    check_against_oracle(spec, x, w, None, mask, 0)
+    assert run_form(spec, x, w, None, mask, 0)[2] == asx.FORM_WINDOW_PATCH
+
+
+def test_tiny_integer_case_is_bit_exact_and_equals_row_gather():
+    """Small integers: every product and sum is exact, so both forms must reproduce the oracle exactly."""
+    spec = wl.LayerSpec("pint", 64, 16, 3, 3, 1, 1, 9, 8, 2, 50, 1, "smallint", 777)
+    x, w, b, mask = make_problem(spec)
+    ref = oracle.masked_conv(x, w, b, mask, 1, 1, True).reshape(spec.M, spec.C_out)
+    ya, _, fa = run_form(spec, x, w, b, mask, asx.ACT_RELU)
+    yb, _, fb = run_form(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_ROW_GATHER)
+    assert fa == asx.FORM_WINDOW_PATCH and fb == asx.FORM_ROW_GATHER_TMA
+    assert np.array_equal(ya, ref) and np.array_equal(yb, ref)
+
+
+def test_more_tiles_than_the_row_coordinate_ring():
+    """Enough kept rows that a block works through more tiles than the ring of decoded tiles holds
+    (8 per block): the row-coordinate warp, the ring's reuse and the patch buffers' turn-taking all run.
+    Checked on sampled rows (the oracle computes them one by one)."""
+    spec = spec_of("p_many", 64, 64, 3, 3, 1, 56, 56, 64, 10, 4, seed=60)      # 180 000 kept rows: more than 9 tiles per block
+    x, w, b, mask = make_problem(spec)
+    rng = np.random.default_rng(5)
+    sel = np.sort(rng.choice(spec.M, 1536, replace=False)).astype(np.int64)
+    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU, rows_sel=sel)
+    y, bits, form = run_form(spec, x, w, b, mask, asx.ACT_RELU)
+    assert form == asx.FORM_WINDOW_PATCH
+    # and the whole tensor equals the row-gather form to within two bf16 roundings of the same sums
+    y2, bits2, form2 = run_form(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_ROW_GATHER)
+    assert form2 == asx.FORM_ROW_GATHER_TMA
+    assert np.array_equal(bits == 0, bits2 == 0) or np.abs(y - y2).max() < 0.1
+    assert np.abs(y - y2).max() <= 2 * max_abs_tol(spec.K, oracle.bf16_round(x), oracle.bf16_round(w))
+    assert np.linalg.norm(y - y2) / np.linalg.norm(y2) <= REL_FROB_TOL
+
+
+def test_residual_add():
+    spec = spec_of("p_res", 64, 64, 3, 3, 1, 14, 14, 3, 50, 4, seed=70)
+    x, w, b, mask = make_problem(spec)
+    rng = np.random.default_rng(9)
+    res = rng.standard_normal((spec.M, spec.C_out)).astype(np.float32)
+    resd = to_dev_bf16(res.reshape(spec.Nb, spec.Ho, spec.Wo, spec.C_out))
+    layer = asx.MaskedConvLayer(64, 64, 3, 3, 1, 1)
+    layer.set_mask(mask)
+    layer.set_residual(resd)
+    out = layer.run(to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda(), flags=asx.ACT_RELU)
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0 and layer.last_run_form() == asx.FORM_WINDOW_PATCH
+    layer.close()
+    pre = oracle.masked_conv(x, w, b, mask, 1, 1, False).reshape(spec.M, spec.C_out)
+    fm = np.tile(mask, spec.Nb).astype(bool)
+    ref = np.where(fm[:, None], np.maximum(pre + oracle.bf16_round(res).astype(np.float64), 0.0), 0.0)
+    got = out.float().cpu().numpy().astype(np.float64).reshape(spec.M, spec.C_out)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= REL_FROB_TOL
+    assert np.abs(got - ref).max() <= max_abs_tol(spec.K, oracle.bf16_round(x), oracle.bf16_round(w)) + 2.0 ** -7 * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("pct", [75, 90, 97])
+def test_sparse_masks_cut_into_short_tiles(pct):
+    """At high sparsity the windows of 128 kept rows span more input rows than a patch buffer holds, so
+    the host cuts shorter tiles (or the planner prefers the row gather): the result must not depend on it."""
+    spec = spec_of("p_sparse", 64, 64, 3, 3, 1, 56, 56, 2, pct, 1, seed=80 + pct)
+    x, w, b, mask = make_problem(spec)
+    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU)
+    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_ROW_GATHER)
+    assert run_form(spec, x, w, b, mask, asx.ACT_RELU)[2] in (asx.FORM_WINDOW_PATCH, asx.FORM_ROW_GATHER_TMA)
+
+
+def test_wide_rows_cut_into_short_tiles():
+    """112 x 112 x 64: one padded input row is 15 KB, a patch buffer holds five of them, so most tiles are
+    cut before they reach 128 rows."""
+    spec = spec_of("p_wide", 64, 32, 3, 3, 1, 112, 112, 1, 30, 2, seed=95)
+    x, w, b, mask = make_problem(spec)
+    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU | asx.RECOMPACT)
+
+
+def test_device_masks_take_the_row_gather():
+    """A mask given as a device pointer is not known to the host: no window-patch plan."""
+    spec = spec_of("p_devmask", 64, 64, 3, 3, 1, 20, 20, 2, 30, 1, seed=90)
+    x, w, b, mask = make_problem(spec)
+    layer = asx.MaskedConvLayer(64, 64, 3, 3, 1, 1)
+    layer.set_mask(torch.from_numpy(mask).cuda())
+    out = layer.run(to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda(), flags=asx.ACT_RELU | asx.RECOMPACT)
+    torch.cuda.synchronize()
+    assert layer.last_run_form() == asx.FORM_ROW_GATHER_TMA
+    layer.close()
+    ref = oracle.masked_conv(x, w, b, mask, 1, 1, True).reshape(spec.M, spec.C_out)
+    got = out.float().cpu().numpy().astype(np.float64).reshape(spec.M, spec.C_out)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= REL_FROB_TOL
