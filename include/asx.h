@@ -60,11 +60,15 @@ enum {
                               network of Section 4); not together with ASX_ACT_RELU (ASX_ERR_INVALID_ARG) */
     ASX_F32 = 64,          /* x, w and y are fp32, the storage type of Appendix A, Algorithm 2 (its sizeof(float));
                               the products run on the tensor cores in TF32, see asx_run */
-    ASX_IMPL_ROW_GATHER = 128  /* always build the lowered rows by gathering every filter tap of every kept row
+    ASX_IMPL_ROW_GATHER = 128, /* always build the lowered rows by gathering every filter tap of every kept row
                               separately (the general form of the producer), also where the library would load a
                               tile's window range once and cut the taps out of it (stride-1 layers with several
                               taps and C_in % 64 == 0 whose mask came from host memory).  Same results up to
                               summation order; a tuning and test switch */
+    ASX_IMPL_WINDOW_PATCH = 256  /* the opposite switch: take the window-range form wherever it can run, also where
+                              the library's cost estimate prefers the row gather.  Layers it cannot run
+                              (see ASX_IMPL_ROW_GATHER) are not affected.  Not together with ASX_IMPL_ROW_GATHER
+                              (ASX_ERR_INVALID_ARG) */
 };
 
 /* Human-readable name of a status code; never NULL; static storage. */
@@ -171,7 +175,7 @@ asx_status asx_recompact(asx_layer* layer, void* cuda_stream);
  *   y    : device, bf16 [Nb][Ho][Wo][C_out], Ho = (H + 2*pad - kh)/stride + 1 (Wo alike);
  *          16-byte aligned when C_out % 8 == 0, else 2-byte; must not overlap x.
  *   flags: OR of ASX_ACT_RELU or ASX_ACT_SILU, ASX_RECOMPACT, ASX_IMPL_NAIVE, ASX_OUT_COMPACT, ASX_IN_COMPACT, ASX_F32,
- *          ASX_IMPL_ROW_GATHER.
+ *          ASX_IMPL_ROW_GATHER or ASX_IMPL_WINDOW_PATCH.
  *          Dropped positions are 0 under every activation (each maps 0 to 0; no bias is added there).  With
  *          ASX_OUT_COMPACT y is bf16 [Nb*P'][C_out] (P' = kept entries of the mask, which must then be
  *          shared by the batch); with ASX_IN_COMPACT x is bf16 [Nb*P'_in][C_in] (see asx_set_input_mask).

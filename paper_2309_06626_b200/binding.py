@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libasx.so")
 _lib = None
 
-ACT_RELU, RECOMPACT, IMPL_NAIVE, OUT_COMPACT, IN_COMPACT, ACT_SILU, F32, IMPL_ROW_GATHER = 1, 2, 4, 8, 16, 32, 64, 128
+ACT_RELU, RECOMPACT, IMPL_NAIVE, OUT_COMPACT, IN_COMPACT, ACT_SILU, F32, IMPL_ROW_GATHER, IMPL_WINDOW_PATCH = 1, 2, 4, 8, 16, 32, 64, 128, 256
 
 # every symbol include/asx.h declares
 EXPORTS = (

@@ -407,7 +407,8 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
 {
     if (L == nullptr || x == nullptr || w == nullptr || y == nullptr) return ASX_ERR_INVALID_ARG;
     if (Nb < 1 || H < 1 || W < 1) return ASX_ERR_INVALID_ARG;
-    if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE | ASX_OUT_COMPACT | ASX_IN_COMPACT | ASX_ACT_SILU | ASX_F32 | ASX_IMPL_ROW_GATHER)) return ASX_ERR_INVALID_ARG;
+    if (flags & ~(ASX_ACT_RELU | ASX_RECOMPACT | ASX_IMPL_NAIVE | ASX_OUT_COMPACT | ASX_IN_COMPACT | ASX_ACT_SILU | ASX_F32 | ASX_IMPL_ROW_GATHER | ASX_IMPL_WINDOW_PATCH)) return ASX_ERR_INVALID_ARG;
+    if ((flags & ASX_IMPL_ROW_GATHER) && (flags & ASX_IMPL_WINDOW_PATCH)) return ASX_ERR_INVALID_ARG;
     const bool f32 = (flags & ASX_F32) != 0;
     const int ES = f32 ? 4 : 2;                 // bytes per element of x, w and y
     const int EPC = 16 / ES;                    // elements per 16-byte chunk
@@ -642,7 +643,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         }
         if (L->tiles_rows > 0 && L->tiles_rows == est_rows) {
             plan_patch_cost(g, L->num_sms, (long long)(L->host_tiles.size() / 2), &pplan);
-            use_patch = pplan.est_cost_us <= plan.est_cost_us;
+            use_patch = pplan.est_cost_us <= plan.est_cost_us || (flags & ASX_IMPL_WINDOW_PATCH);
         }
     }
     if (plan.ksplit > 1 && !use_patch) {

@@ -564,14 +564,15 @@ bool plan_patch(const ConvGeom& g, int fused_list_rows, PatchPlan* plan)
 
 void plan_patch_cost(const ConvGeom& g, int num_sms, long long n_mtiles, PatchPlan* plan)
 {
-    // Estimated duration, in the terms of the row-gather planner: a pipeline stage of G taps costs the
-    // issuing thread about 0.12 microseconds of waits and commits plus the tensor-core time of its
-    // 4 G instructions (BN / 2 clocks each); the last tile's epilogue about 0.012 BN.
+    // Estimated duration, in the terms of the row-gather planner and from the same kind of measurement:
+    // a 64-wide k-block of a 128 x BN tile takes about 0.21 + 0.001 BN microseconds here (against
+    // 0.30 + 0.001 BN for the row gather).  Both forms are bound by shared-memory bandwidth: per k-block
+    // this one moves 16 KB of patch reads, the filter slab in and out (BN x 256 bytes) and its share of
+    // the patch, the row gather 32 KB of A rows in and out plus the same slab.
     const long long items = n_mtiles * plan->n_tiles;
     const long long waves = (items + num_sms - 1) / num_sms;
-    const int taps = g.kh * g.kw;
-    const int stages = (taps + plan->G - 1) / plan->G * (g.C_in / 64);
-    const double t_tile = stages * 0.12 + taps * (g.C_in / 64) * 4 * (plan->BN / 2) / 1900.0;
+    const int KB = g.kh * g.kw * (g.C_in / 64);
+    const double t_tile = KB * (0.21 + 0.001 * plan->BN);
     plan->est_cost_us = (double)waves * (t_tile + 0.3) + 0.012 * plan->BN;
 }
 

@@ -64,12 +64,13 @@ def test_window_patch_against_oracle(case, act):
     x, w, b, mask = make_problem(spec)
     layer = asx.MaskedConvLayer(spec.C_in, spec.C_out, spec.kh, spec.kw, 1, spec.pad)
     layer.set_mask(mask)
-    layer.run(to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda(), flags=act)
+    layer.run(to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda(), flags=act | asx.IMPL_WINDOW_PATCH)
     torch.cuda.synchronize()
     assert layer.last_run_form() == asx.FORM_WINDOW_PATCH, "this case is meant to take the window-patch form"
     layer.close()
-    check_against_oracle(spec, x, w, b, mask, act)
-    check_against_oracle(spec, x, w, b, mask, act | asx.RECOMPACT)
+    check_against_oracle(spec, x, w, b, mask, act | asx.IMPL_WINDOW_PATCH)
+    check_against_oracle(spec, x, w, b, mask, act | asx.RECOMPACT | asx.IMPL_WINDOW_PATCH)
+    check_against_oracle(spec, x, w, b, mask, act)                        # whichever form the library picks
 
 
 @pytest.mark.parametrize("kept_rows", [0, 1, 127, 128, 129, 255, 256, 257, "all"])
@@ -81,16 +82,16 @@ def test_tile_boundaries(kept_rows):
         mask[:] = 1
     else:
         mask[np.random.default_rng(kept_rows).permutation(spec.P)[:kept_rows]] = 1
-    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU)
-    y, bits, form = run_form(spec, x, w, b, mask, asx.ACT_RELU)
+    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_WINDOW_PATCH)
+    y, bits, form = run_form(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_WINDOW_PATCH)
     assert form == asx.FORM_WINDOW_PATCH or kept_rows == 0      # with nothing kept there are no tiles to cut
 
 
 def test_per_row_mask():
     spec = spec_of("p_rowmask", 64, 64, 3, 3, 1, 18, 21, 3, 40, 2, seed=50)
     x, w, b, mask = make_problem(spec, per_row=True)
-    check_against_oracle(spec, x, w, None, mask, 0)
-    assert run_form(spec, x, w, None, mask, 0)[2] == asx.FORM_WINDOW_PATCH
+    check_against_oracle(spec, x, w, None, mask, asx.IMPL_WINDOW_PATCH)
+    assert run_form(spec, x, w, None, mask, asx.IMPL_WINDOW_PATCH)[2] == asx.FORM_WINDOW_PATCH
 
 
 def test_tiny_integer_case_is_bit_exact_and_equals_row_gather():
@@ -98,7 +99,7 @@ def test_tiny_integer_case_is_bit_exact_and_equals_row_gather():
     spec = wl.LayerSpec("pint", 64, 16, 3, 3, 1, 1, 9, 8, 2, 50, 1, "smallint", 777)
     x, w, b, mask = make_problem(spec)
     ref = oracle.masked_conv(x, w, b, mask, 1, 1, True).reshape(spec.M, spec.C_out)
-    ya, _, fa = run_form(spec, x, w, b, mask, asx.ACT_RELU)
+    ya, _, fa = run_form(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_WINDOW_PATCH)
     yb, _, fb = run_form(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_ROW_GATHER)
     assert fa == asx.FORM_WINDOW_PATCH and fb == asx.FORM_ROW_GATHER_TMA
     assert np.array_equal(ya, ref) and np.array_equal(yb, ref)
@@ -112,8 +113,8 @@ def test_more_tiles_than_the_row_coordinate_ring():
     x, w, b, mask = make_problem(spec)
     rng = np.random.default_rng(5)
     sel = np.sort(rng.choice(spec.M, 1536, replace=False)).astype(np.int64)
-    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU, rows_sel=sel)
-    y, bits, form = run_form(spec, x, w, b, mask, asx.ACT_RELU)
+    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_WINDOW_PATCH, rows_sel=sel)
+    y, bits, form = run_form(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_WINDOW_PATCH)
     assert form == asx.FORM_WINDOW_PATCH
     # and the whole tensor equals the row-gather form to within two bf16 roundings of the same sums
     y2, bits2, form2 = run_form(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_ROW_GATHER)
@@ -132,7 +133,7 @@ def test_residual_add():
     layer = asx.MaskedConvLayer(64, 64, 3, 3, 1, 1)
     layer.set_mask(mask)
     layer.set_residual(resd)
-    out = layer.run(to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda(), flags=asx.ACT_RELU)
+    out = layer.run(to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda(), flags=asx.ACT_RELU | asx.IMPL_WINDOW_PATCH)
     torch.cuda.synchronize()
     assert layer.device_status() == 0 and layer.last_run_form() == asx.FORM_WINDOW_PATCH
     layer.close()
@@ -152,7 +153,8 @@ def test_sparse_masks_cut_into_short_tiles(pct):
     x, w, b, mask = make_problem(spec)
     check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU)
     check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_ROW_GATHER)
-    assert run_form(spec, x, w, b, mask, asx.ACT_RELU)[2] in (asx.FORM_WINDOW_PATCH, asx.FORM_ROW_GATHER_TMA)
+    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_WINDOW_PATCH)
+    assert run_form(spec, x, w, b, mask, asx.ACT_RELU | asx.IMPL_WINDOW_PATCH)[2] == asx.FORM_WINDOW_PATCH
 
 
 def test_wide_rows_cut_into_short_tiles():
@@ -160,7 +162,7 @@ def test_wide_rows_cut_into_short_tiles():
     cut before they reach 128 rows."""
     spec = spec_of("p_wide", 64, 32, 3, 3, 1, 112, 112, 1, 30, 2, seed=95)
     x, w, b, mask = make_problem(spec)
-    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU | asx.RECOMPACT)
+    check_against_oracle(spec, x, w, b, mask, asx.ACT_RELU | asx.RECOMPACT | asx.IMPL_WINDOW_PATCH)
 
 
 def test_device_masks_take_the_row_gather():
