@@ -285,7 +285,7 @@ def run_ours(args):
     import torch.distributed as dist
     import paper_2309_06626_b200 as asx
     from paper_2309_06626_b200 import build as asx_build
-    from paper_2309_06626_b200.dist_util import max_over_ranks, whole_job_rate
+    from paper_2309_06626_b200.dist_util import max_over_ranks, shard_batch, whole_job_rate
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -318,6 +318,14 @@ def run_ours(args):
         specs = [s for s in specs if any(s.name.startswith(p) for p in args.only.split(","))]
         if not specs:
             raise SystemExit(f"--only {args.only}: no such layer")
+    strong = (args.scaling == "strong" and world > 1)
+    if strong:
+        # the batch of every layer is split across the ranks (images [lo, hi) of each); the masks are
+        # shared by the images, so every rank keeps the whole mask and kept-row list
+        shards = [shard_batch(s.Nb, rank, world) for s in specs]
+        if any(hi <= lo for lo, hi in shards):
+            raise SystemExit("--scaling strong needs at least one image per rank in every layer")
+        specs = [wl.with_batch(s, hi - lo) for s, (lo, hi) in zip(specs, shards)]
     score = None
     if args.mask == "scores":
         score = wl.make_score(args.config, max(s.H for s in specs), max(s.W for s in specs))
@@ -454,7 +462,13 @@ def run_ours(args):
 
     flops_step = sum(L.flops for L in layers)
     dense_flops_step = sum(L.flops_dense for L in layers)
-    value = whole_job_rate(flops_step, ms_step, world) / 1e12
+    if strong:     # the ranks' shards differ by at most one image: sum them instead of multiplying
+        tot = torch.tensor([float(flops_step), float(dense_flops_step)], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tot)
+        job_flops, job_dense_flops = float(tot[0].item()), float(tot[1].item())
+    else:
+        job_flops, job_dense_flops = world * flops_step, world * dense_flops_step
+    value = (job_flops / (ms_step * 1e-3) if strong else whole_job_rate(flops_step, ms_step, world)) / 1e12
 
     per_layer_ms = [statistics.median(row[i][0].elapsed_time(row[i][1]) for row in probe_events)
                     for i in range(len(layers))]
@@ -543,7 +557,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - tw0) * 1e3 / Ke
     e2e_ms = max_over_ranks(e2e_ms, device="cuda")
-    e2e_val = whole_job_rate(flops_step, e2e_ms, world) / 1e12
+    e2e_val = job_flops / (e2e_ms * 1e-3) / 1e12
     t_gpu_end = time.time()
 
     if rank != 0:
@@ -682,7 +696,7 @@ def run_ours(args):
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": K,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "strong" if strong else "weak",
         "vs_baseline": None, "dtype": "tf32" if f32 else "bf16", "data": "synthetic",
         "config": {"workload": workload_name(args.config) + (f" [only {args.only}]" if args.only else ""),
                    "layers": len(layers),
@@ -729,7 +743,7 @@ def run_ours(args):
                            + (" x 1.1/2.25, the nominal ratio of the dense TF32 and bf16 rates" if f32 else ""),
             # the other half of the metric and the side legs, kept here so that they are stored with the record
             "metric_parts": {
-                "dense_equivalent_tflops": world * dense_flops_step / (ms_step * 1e-3) / 1e12,
+                "dense_equivalent_tflops": job_dense_flops / (ms_step * 1e-3) / 1e12,
                 "speedup_vs_sparsity0": (ms_dense / ms_step) if ms_dense else None,
                 "ms_per_step_sparsity0": ms_dense,
                 "speedup_vs_cudnn_dense": (cudnn_ms / ms_step) if cudnn_ms else None,
@@ -779,6 +793,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-cudnn", action="store_true")
     ap.add_argument("--only", default="", help="comma-separated layer-name prefixes: run a sub-stack (profiling)")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="with N > 1 ranks: every rank runs the whole batch (weak, the default) or its share of the images (strong)")
     ap.add_argument("--no-fork-proj", action="store_true",
                     help="keep the 1x1 projections of down-sampling blocks in line instead of on a graph branch")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")

@@ -131,7 +131,7 @@ asx_status asx_set_mask_from_scores(asx_layer* layer, const float* score, int H0
 
 /*
  * Layer chaining without re-densifying.  The paper expands every masked layer's output back to the
- * dense shape only because "the subsequent layer assumes dense activation" (Section 3.2, stage
+ * dense shape only because the layer that follows expects an ordinary dense tensor (Section 3.2, stage
  * iii) and names that post-processing as one of its two overheads (Section 4.3).  Here a layer run
  * with ASX_OUT_COMPACT writes row j of the kept list of image n at y[n*P' + j][0..C_out) and writes
  * nothing else, and the layer that consumes it is run with ASX_IN_COMPACT after being told the
@@ -243,6 +243,18 @@ asx_status asx_last_run_form(const asx_layer* layer, int* form);
  */
 asx_status asx_set_wait_limit(asx_layer* layer, int64_t cycles);
 
+/*
+ * Test hook for the bounded waits (no counterpart in the paper).  Layers with few kept rows and a long
+ * reduction share a tile's k-blocks between thread blocks, which meet at a per-tile arrival counter in
+ * the layer's workspace.  This call overwrites the arrival counter of output tile `tile` with `value`
+ * (in stream order); a value the arrivals can never lift to the number of shares makes the waiting
+ * blocks run into their wait limit, which is how the time-out path is exercised from the host without
+ * faulting or hanging the GPU.  ASX_ERR_UNSUPPORTED if the layer's last plan did not share k-blocks (no
+ * counters exist), ASX_ERR_INVALID_ARG for a tile outside the workspace.  asx_last_device_status puts
+ * the counters back to zero after a reported time-out.
+ */
+asx_status asx_debug_set_split_counter(asx_layer* layer, int64_t tile, int32_t value, void* cuda_stream);
+
 /* Free the layer and the device memory it owns.  NULL is allowed. */
 asx_status asx_destroy(asx_layer* layer);
 
@@ -264,8 +276,9 @@ asx_status asx_compact(const uint8_t* mask_dev, int64_t rows, int32_t* kept_dev,
                        int32_t* count_dev, void* scratch_dev, int64_t scratch_bytes,
                        void* cuda_stream);
 /* Waits for `cuda_stream`, then reports the status word the last asx_compact left in this scratch
- * buffer: ASX_OK, or ASX_ERR_TIMEOUT if a kernel gave up in a bounded wait (the compaction kernels
- * have no such wait any more, so this reports ASX_OK after any completed call). */
+ * buffer: ASX_OK, or ASX_ERR_TIMEOUT if a kernel gave up in a bounded wait.  The compaction kernels
+ * no longer contain any wait on another block, so after a completed call this always reports
+ * ASX_OK; the entry point is kept so that callers built against it keep linking. */
 asx_status asx_compact_status(const void* scratch_dev, void* cuda_stream);
 
 /*
@@ -295,10 +308,13 @@ asx_status asx_mask_from_activation(const void* x_dev, int64_t rows, int C, uint
  *          asx_compact.
  * The array (about 32 KB) is part of the library image on every GPU that loads it.  The first
  * call on each device looks up the array's device address; make that first call outside any
- * stream capture.  All calls on a device share the one array: it is cleared on the stream at
- * the start of each call, and two calls that may overlap on the GPU (different streams without
- * an ordering between them) race on it and give undefined lists.  A bounded-wait timeout inside
- * the kernel cannot be queried through this entry point.
+ * stream capture, and do not let two host threads make a device's first call at the same moment
+ * (both would look the address up; they store the same value).  All calls on a device share the
+ * one array and it keeps the last call's contents: every call overwrites, in stream order, each
+ * word it later reads, so nothing needs clearing, but two calls that may overlap on the GPU
+ * (different streams without an ordering between them) race on it and give undefined lists.
+ * The mask may have been written by the kernel launched just before on the same stream (for
+ * instance asx_mask_from_activation): the kernels read it only after that kernel has finished.
  */
 #define ASX_COMPACT_STATIC_MAX_ROWS (1 << 24)
 asx_status asx_compact_static(const uint8_t* mask_dev, int64_t rows, int32_t* kept_dev,

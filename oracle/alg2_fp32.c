@@ -4,9 +4,10 @@
  * path).
  *
  * Appendix A, Algorithm 2 and Section 3.2 describe three stages for one image:
- *   (i)   an indirection buffer that holds, for every output position whose mask entry is 1 and in
- *         raster order, the pointers to the input pixels under the filter window; positions with
- *         mask 0 get no entry, so the buffer has P' = sum(mask) rows of kh*kw pointers;
+ *   (i)   an indirection table that holds, for every output position whose mask entry is 1 and in
+ *         raster order, where the input pixels under the filter window are (the paper keeps
+ *         pointers, this file element offsets); positions with mask 0 get no entry, so the table
+ *         has P' = sum(mask) rows of kh*kw entries;
  *   (ii)  the unmodified dense GEMM over that reduced range: row r of the compact output is the
  *         product of the gathered window of kept position r with the filter matrix, plus the bias
  *         (the engine's fp32 arithmetic; the activation is applied here, on computed rows only);
@@ -16,7 +17,7 @@
  *         decremented, so no row is overwritten before it has been moved.
  *
  * Readings: the printed index out_y * output_height + out_x is taken as the row-major position
- * out_y * output_width + out_x; padding taps point at a row of zeros; the mask is shared by the
+ * out_y * output_width + out_x; padding taps are marked and contribute zeros; the mask is shared by the
  * images of a batch; the GEMM is a plain triple loop (the paper uses the engine's micro-kernels,
  * whose blocking is not part of the method).
  */
@@ -24,57 +25,63 @@
 #include <stdlib.h>
 #include <string.h>
 
-/* Stage (i): pointers of the kept windows of one image.  Returns P'. */
-static int64_t indirection_init(const float *x_img, int H, int W, int C_in, int kh, int kw, int stride, int pad,
-                                int Ho, int Wo, const uint8_t *mask, const float *zero_row, const float **ind)
+/* Stage (i): the window table of one image.  Entry (r, t) is the element offset, within the image,
+ * of the input pixel under filter tap t of the r-th kept position (kept positions in ascending flat
+ * order), or -1 where the tap falls into the padding.  Returns the number of kept positions. */
+static int64_t build_window_table(int H, int W, int C_in, int kh, int kw, int stride, int pad, int Wo, int64_t P,
+                                  const uint8_t *mask, int64_t *table)
 {
-    int64_t index = 0;
-    for (int out_y = 0; out_y < Ho; ++out_y)
-        for (int out_x = 0; out_x < Wo; ++out_x) {
-            if (mask[(int64_t)out_y * Wo + out_x] == 0) continue;
-            for (int ky = 0; ky < kh; ++ky)
-                for (int kx = 0; kx < kw; ++kx) {
-                    const int iy = out_y * stride - pad + ky, ix = out_x * stride - pad + kx;
-                    const int inside = iy >= 0 && iy < H && ix >= 0 && ix < W;
-                    ind[index * kh * kw + ky * kw + kx] = inside ? x_img + ((int64_t)iy * W + ix) * C_in : zero_row;
-                }
-            ++index;
+    const int taps = kh * kw;
+    int64_t n_kept = 0;
+    for (int64_t p = 0; p < P; ++p) {
+        if (!mask[p]) continue;                       /* a dropped position gets no entry */
+        const int top = (int)(p / Wo) * stride - pad, left = (int)(p % Wo) * stride - pad;
+        int64_t *entry = table + n_kept * taps;
+        for (int t = 0; t < taps; ++t) {
+            const int iy = top + t / kw, ix = left + t % kw;
+            entry[t] = (iy >= 0 && iy < H && ix >= 0 && ix < W) ? ((int64_t)iy * W + ix) * C_in : -1;
         }
-    return index;
+        ++n_kept;
+    }
+    return n_kept;
 }
 
-/* Stage (ii): dense product over the kept rows, written compactly at the start of `out`. */
-static void gemm_reduced(const float **ind, int64_t kept, int taps, int C_in, const float *w, const float *bias,
-                         int C_out, int relu, float *out)
+/* Stage (ii): the dense product restricted to the kept rows; compact row r goes to rows[r]. */
+static void product_on_kept_rows(const float *x_img, const int64_t *table, int64_t n_kept, int taps, int C_in,
+                                 const float *w, const float *bias, int C_out, int relu, float *rows)
 {
 #pragma omp parallel for schedule(static)
-    for (int64_t r = 0; r < kept; ++r)
+    for (int64_t r = 0; r < n_kept; ++r)
         for (int co = 0; co < C_out; ++co) {
             float acc = bias ? bias[co] : 0.0f;
             for (int t = 0; t < taps; ++t) {
-                const float *px = ind[r * taps + t];
+                const int64_t off = table[r * taps + t];
+                if (off < 0) continue;                /* padding contributes zeros */
+                const float *px = x_img + off;
                 const float *wt = w + ((int64_t)co * taps + t) * C_in;
                 for (int ci = 0; ci < C_in; ++ci) acc += px[ci] * wt[ci];
             }
-            out[r * C_out + co] = (relu && acc < 0.0f) ? 0.0f : acc;
+            rows[r * C_out + co] = (relu && acc < 0.0f) ? 0.0f : acc;
         }
 }
 
-/* Stage (iii): reverse in-place expansion of the compact rows to the dense output of one image. */
-static void post_process(float *out, int Ho, int Wo, int C_out, const uint8_t *mask, int64_t kept)
+/* Stage (iii): the compact rows occupy the first n_kept rows of the image's output; spread them to
+ * their positions in place.  Going from the last position down, the row still to be placed (`src`)
+ * never lies above its destination, so a row is moved before anything can overwrite it; dropped
+ * positions are cleared on the way. */
+static void expand_in_place(float *out, int64_t P, int C_out, const uint8_t *mask, int64_t n_kept)
 {
-    const size_t outch_size = (size_t)C_out * sizeof(float);
-    int64_t id = kept - 1;
-    for (int out_y = Ho - 1; out_y >= 0; --out_y)
-        for (int out_x = Wo - 1; out_x >= 0; --out_x) {
-            const int64_t pos = (int64_t)out_y * Wo + out_x;
-            if (mask[pos] == 0) {
-                memset(out + pos * C_out, 0, outch_size);
-            } else {
-                if (pos != id) memmove(out + pos * C_out, out + id * C_out, outch_size);
-                --id;
-            }
+    const size_t row_bytes = (size_t)C_out * sizeof(float);
+    int64_t src = n_kept;                             /* rows [0, src) are still compact */
+    for (int64_t p = P; p-- > 0;) {
+        float *dst = out + p * C_out;
+        if (mask[p]) {
+            --src;
+            if (src != p) memmove(dst, out + src * C_out, row_bytes);
+        } else {
+            memset(dst, 0, row_bytes);
         }
+    }
 }
 
 /*
@@ -89,17 +96,15 @@ int asxo_alg2_fp32(const float *x, int Nb, int H, int W, int C_in, const float *
     const int Ho = (H + 2 * pad - kh) / stride + 1, Wo = (W + 2 * pad - kw) / stride + 1;
     const int taps = kh * kw;
     const int64_t P = (int64_t)Ho * Wo;
-    float *zero_row = (float *)calloc((size_t)C_in, sizeof(float));
-    const float **ind = (const float **)malloc((size_t)P * taps * sizeof(const float *));
-    if (!zero_row || !ind) { free(zero_row); free((void *)ind); return 1; }
+    int64_t *table = (int64_t *)malloc((size_t)P * taps * sizeof(int64_t));
+    if (!table) return 1;
     for (int n = 0; n < Nb; ++n) {
         const float *x_img = x + (int64_t)n * H * W * C_in;
         float *y_img = y + (int64_t)n * P * C_out;
-        const int64_t kept = indirection_init(x_img, H, W, C_in, kh, kw, stride, pad, Ho, Wo, mask, zero_row, ind);
-        gemm_reduced(ind, kept, taps, C_in, w, bias, C_out, relu, y_img);
-        post_process(y_img, Ho, Wo, C_out, mask, kept);
+        const int64_t n_kept = build_window_table(H, W, C_in, kh, kw, stride, pad, Wo, P, mask, table);
+        product_on_kept_rows(x_img, table, n_kept, taps, C_in, w, bias, C_out, relu, y_img);
+        expand_in_place(y_img, P, C_out, mask, n_kept);
     }
-    free(zero_row);
-    free((void *)ind);
+    free(table);
     return 0;
 }

@@ -17,7 +17,7 @@ EXPORTS = (
     "asx_get_kept", "asx_get_kept_host", "asx_get_mask", "asx_last_device_status", "asx_destroy",
     "asx_compact_scratch_bytes", "asx_compact", "asx_compact_status", "asx_compact_static",
     "asx_mask_from_scores", "asx_set_mask_from_scores", "asx_mask_from_activation", "asx_set_input_mask", "asx_set_residual",
-    "asx_last_run_form", "asx_set_wait_limit",
+    "asx_last_run_form", "asx_set_wait_limit", "asx_debug_set_split_counter",
 )
 COMPACT_STATIC_MAX_ROWS = 1 << 24
 FORM_NONE, FORM_NAIVE, FORM_ROW_GATHER_COPY, FORM_ROW_GATHER_TMA, FORM_WINDOW_PATCH = 0, 1, 2, 3, 4
@@ -64,6 +64,7 @@ def lib():
         L.asx_set_residual.argtypes = [vp, vp]
         L.asx_last_run_form.argtypes = [vp, ctypes.POINTER(ci)]
         L.asx_set_wait_limit.argtypes = [vp, i64]
+        L.asx_debug_set_split_counter.argtypes = [vp, i64, ctypes.c_int32, vp]
         L.asx_mask_from_activation.argtypes = [vp, i64, ci, vp, vp]
         L.asx_mask_from_scores.argtypes = [vp, ci, ci, ci, ci, ctypes.c_double, vp]
         L.asx_set_mask_from_scores.argtypes = [vp, vp, ci, ci, ci, ci, ctypes.c_double, vp]

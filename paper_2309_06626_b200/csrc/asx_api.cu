@@ -128,7 +128,7 @@ asx_status ensure_mask_buffers(asx_layer* L, int64_t rows)
 
 asx_status run_compaction(asx_layer* L, cudaStream_t st)
 {
-    return from_cuda(launch_compact(L->d_mask, L->rows, L->d_kept, L->d_small, L->d_scratch, st));
+    return from_cuda(launch_compact(L->d_mask, L->rows, L->d_kept, L->d_small, L->d_scratch, st, true));
 }
 
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", 2011).
@@ -793,6 +793,18 @@ asx_status asx_set_wait_limit(asx_layer* L, int64_t cycles)
     return ASX_OK;
 }
 
+asx_status asx_debug_set_split_counter(asx_layer* L, int64_t tile, int32_t value, void* cuda_stream)
+{
+    if (L == nullptr) return ASX_ERR_INVALID_ARG;
+    if (L->d_wscnt == nullptr || L->wscnt_ints == 0) return ASX_ERR_UNSUPPORTED;
+    if (tile < 0 || (size_t)(2 * tile) >= L->wscnt_ints) return ASX_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // the value is copied out of this frame before the call returns (pageable source)
+    if (cudaMemcpyAsync(L->d_wscnt + 2 * tile, &value, sizeof(value), cudaMemcpyHostToDevice, st) != cudaSuccess) return ASX_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return ASX_ERR_CUDA;
+    return ASX_OK;
+}
+
 asx_status asx_destroy(asx_layer* L)
 {
     if (L == nullptr) return ASX_OK;
@@ -820,7 +832,7 @@ asx_status asx_compact(const uint8_t* mask_dev, int64_t rows, int32_t* kept_dev,
     if (reinterpret_cast<uintptr_t>(scratch_dev) & 7) return ASX_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(kept_dev) & 3) || (reinterpret_cast<uintptr_t>(count_dev) & 3)) return ASX_ERR_ALIGN;
     return from_cuda(launch_compact(mask_dev, rows, kept_dev, count_dev, scratch_dev,
-                                    static_cast<cudaStream_t>(cuda_stream)));
+                                    static_cast<cudaStream_t>(cuda_stream), false));
 }
 
 asx_status asx_mask_from_activation(const void* x_dev, int64_t rows, int C, uint8_t* mask_dev, void* cuda_stream)

@@ -47,8 +47,10 @@ constexpr int COMPACT_THREADS = 256;
 constexpr int COMPACT_PER_THREAD = 16;
 constexpr int COMPACT_TILE = COMPACT_THREADS * COMPACT_PER_THREAD;
 int64_t compact_scratch_bytes(int64_t rows);
+// mask_written_by_copies_only: the mask buffer is never written by a kernel (a layer's own copy), so
+// the write pass may read it before its dependency wait; false for a caller's buffer.
 cudaError_t launch_compact(const uint8_t* mask, int64_t rows, int32_t* kept, int32_t* count,
-                           void* scratch, cudaStream_t st);
+                           void* scratch, cudaStream_t st, bool mask_written_by_copies_only);
 
 // ---- debug reference kernels (naive.cu)
 cudaError_t launch_naive(const ConvGeom& g, const void* x, const void* w, const float* bias, void* y,

@@ -14,7 +14,7 @@ namespace asx {
 namespace {
 
 struct ScratchHeader {       // first 8 bytes of the scratch; the tile counts follow
-    unsigned int ticket;     // unused by the kernels (kept zero)
+    unsigned int reserved;   // kept zero
     int error;               // device status word of the compaction (kept zero: nothing here can time out)
 };
 
@@ -46,7 +46,7 @@ __device__ __forceinline__ void load_tile_flags(const uint8_t* __restrict__ mask
         const long long first = tile_first + (long long)sub * COMPACT_TILE + (long long)tid * COMPACT_PER_THREAD;
         fast[sub] = aligned && first + COMPACT_PER_THREAD <= rows;
         raw[sub] = make_uint4(0, 0, 0, 0);
-        if (fast[sub]) raw[sub] = __ldg(reinterpret_cast<const uint4*>(mask + first));
+        if (fast[sub]) raw[sub] = __ldcg(reinterpret_cast<const uint4*>(mask + first));     // past L1: a kernel may have written the mask
     }
 #pragma unroll
     for (int sub = 0; sub < COMPACT_SUB; ++sub) {
@@ -57,7 +57,7 @@ __device__ __forceinline__ void load_tile_flags(const uint8_t* __restrict__ mask
                 (nonzero_bytes4(raw[sub].w) << 12);
         } else {
             for (int j = 0; j < COMPACT_PER_THREAD; ++j)
-                if (first + j < rows && mask[first + j] != 0) f |= 1u << j;
+                if (first + j < rows && __ldcg(mask + first + j) != 0) f |= 1u << j;
         }
         flags[sub] = f;
     }
@@ -138,7 +138,7 @@ compact_scan_tiles_kernel(unsigned* __restrict__ tile_count, int num_tiles, int3
     }
     if (tid == 0) {
         *count = (int32_t)s_carry;
-        hdr->ticket = 0;                   // a status query must find a clean word
+        hdr->reserved = 0;                   // a status query must find a clean word
         hdr->error = 0;
     }
 }
@@ -146,6 +146,12 @@ compact_scan_tiles_kernel(unsigned* __restrict__ tile_count, int num_tiles, int3
 // Pass 3: the indices of a 4096-row sub-tile are put in order in shared memory and copied to the list
 // with full-width stores (direct stores of each 32-row ballot word's indices, without the staging,
 // write half-filled lines and were 12 % slower; 16-byte stores from the unaligned staging buffer 3 %).
+// EARLY_MASK: the mask is only ever written by stream-ordered copies (a layer's own copy of its mask), so
+// the tile's mask bytes may be loaded and scanned before the dependency wait, while the passes before
+// still run.  A caller's mask buffer may have been written by the kernel just before this call (a
+// data-dependent mask), which, launched as a programmatic predecessor, can still be storing it: then the
+// load waits like everything else.
+template <bool EARLY_MASK>
 __global__ void __launch_bounds__(COMPACT_THREADS, 8)
 compact_write_kernel(const uint8_t* __restrict__ mask, long long rows, int32_t* __restrict__ kept,
                      const unsigned* __restrict__ tile_offset)
@@ -156,7 +162,8 @@ compact_write_kernel(const uint8_t* __restrict__ mask, long long rows, int32_t* 
     ptx::grid_launch_dependents();
     const long long tile_first = (long long)blockIdx.x * COMPACT_BIG_TILE;
     unsigned flags[COMPACT_SUB];
-    load_tile_flags(mask, rows, tile_first, tid, flags);      // the mask is not written by the passes before
+    if (!EARLY_MASK) ptx::grid_dependency_wait();
+    load_tile_flags(mask, rows, tile_first, tid, flags);
     int mine[COMPACT_SUB], incl[COMPACT_SUB];
 #pragma unroll
     for (int sub = 0; sub < COMPACT_SUB; ++sub) {
@@ -170,7 +177,7 @@ compact_write_kernel(const uint8_t* __restrict__ mask, long long rows, int32_t* 
         incl[sub] = v;
         if (lane == 31) s_warp_total[sub][warp] = v;
     }
-    ptx::grid_dependency_wait();          // the offsets come from the pass before; the list may still be read
+    if (EARLY_MASK) ptx::grid_dependency_wait();          // the offsets come from the pass before; the list may still be read
     // Read past L1: this block was launched while the passes before were running, L1 is not
     // invalidated in between, and the SM may hold the line as the counting pass left it (a block of the
     // first wave runs on the SM where the counting block of the same tile wrote that word).
@@ -217,12 +224,12 @@ compact_small_kernel(const uint8_t* __restrict__ mask, int rows, int32_t* __rest
     unsigned flags = 0;
     const bool aligned = (reinterpret_cast<uintptr_t>(mask) & 15) == 0;
     if (aligned && first + COMPACT_PER_THREAD <= rows) {
-        const uint4 v = *reinterpret_cast<const uint4*>(mask + first);
+        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(mask + first));      // past L1: a kernel may have written the mask
         flags = nonzero_bytes4(v.x) | (nonzero_bytes4(v.y) << 4) | (nonzero_bytes4(v.z) << 8) |
                 (nonzero_bytes4(v.w) << 12);
     } else {
         for (int j = 0; j < COMPACT_PER_THREAD; ++j)
-            if (first + j < rows && mask[first + j] != 0) flags |= 1u << j;
+            if (first + j < rows && __ldcg(mask + first + j) != 0) flags |= 1u << j;
     }
     const int mine = __popc(flags);
     int incl = mine;
@@ -251,7 +258,7 @@ compact_small_kernel(const uint8_t* __restrict__ mask, int rows, int32_t* __rest
     }
     if (tid == 0) {
         *count = total;
-        if (hdr != nullptr) { hdr->ticket = 0; hdr->error = 0; }     // a status query must find a clean word
+        if (hdr != nullptr) { hdr->reserved = 0; hdr->error = 0; }     // a status query must find a clean word
     }
 }
 
@@ -269,7 +276,7 @@ int64_t compact_scratch_bytes(int64_t rows)
 }
 
 cudaError_t launch_compact(const uint8_t* mask, int64_t rows, int32_t* kept, int32_t* count,
-                           void* scratch, cudaStream_t st)
+                           void* scratch, cudaStream_t st, bool mask_written_by_copies_only)
 {
     auto* hdr = static_cast<ScratchHeader*>(scratch);
     if (rows <= COMPACT_SMALL_MAX_ROWS)
@@ -280,8 +287,11 @@ cudaError_t launch_compact(const uint8_t* mask, int64_t rows, int32_t* kept, int
     cudaError_t e = launch_pdl(compact_count_kernel, dim3(tiles), dim3(COMPACT_THREADS), 0, st, mask, (long long)rows, tile_count);
     if (e == cudaSuccess) e = launch_pdl(compact_scan_tiles_kernel, dim3(1), dim3(1024), 0, st, tile_count, tiles, count, hdr);
     if (e == cudaSuccess)
-        e = launch_pdl(compact_write_kernel, dim3(tiles), dim3(COMPACT_THREADS), 0, st, mask, (long long)rows, kept,
-                       static_cast<const unsigned*>(tile_count));
+        e = mask_written_by_copies_only
+                ? launch_pdl(compact_write_kernel<true>, dim3(tiles), dim3(COMPACT_THREADS), 0, st, mask, (long long)rows, kept,
+                             static_cast<const unsigned*>(tile_count))
+                : launch_pdl(compact_write_kernel<false>, dim3(tiles), dim3(COMPACT_THREADS), 0, st, mask, (long long)rows, kept,
+                             static_cast<const unsigned*>(tile_count));
     return e;
 }
 
@@ -336,7 +346,7 @@ extern "C" asx_status asx_compact_static(const uint8_t* mask_dev, int64_t rows, 
     // launch_compact overwrites every word of the array it later reads (tile counts, header), in
     // stream order, so whatever the previous call left in the array does not matter.
     return asx::launch_compact(mask_dev, rows, kept_dev, count_dev, g_static_scratch_addr[dev],
-                               static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+                               static_cast<cudaStream_t>(cuda_stream), false) == cudaSuccess
                ? ASX_OK
                : ASX_ERR_CUDA;
 }

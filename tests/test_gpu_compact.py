@@ -93,3 +93,38 @@ def test_back_to_back_calls_on_changing_masks():
         ref = oracle.kept_list(m)
         assert int(count.item()) == ref.size
         assert np.array_equal(kept[:ref.size].cpu().numpy(), ref)
+
+
+@pytest.mark.parametrize("rows", [9_000, 1_600_000])
+def test_mask_written_by_the_kernel_just_before(rows):
+    """asx_mask_from_activation -> asx_compact / asx_compact_static into the SAME mask buffer, with a
+    different activation every round and no host synchronisation: the compaction kernels start while
+    the mask kernel may still be storing the mask, and must read it only once it has finished (and
+    not from a stale L1 line of the previous round)."""
+    C = 8
+    rng = np.random.default_rng(rows)
+    st = int(torch.cuda.current_stream().cuda_stream)
+    mask = torch.zeros(rows, dtype=torch.uint8, device="cuda")
+    nb = asx.lib().asx_compact_scratch_bytes(rows)
+    scr = torch.empty((nb + 7) // 8, dtype=torch.int64, device="cuda")
+    rounds, acts, outs = 6, [], []
+    for r in range(rounds):
+        x = np.maximum(rng.standard_normal((rows, C)).astype(np.float32), 0.0)
+        x[rng.random(rows) < (0.2 + 0.1 * r)] = 0.0
+        acts.append(torch.from_numpy(x).to(torch.bfloat16).cuda())
+    for r in range(rounds):
+        k1 = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
+        k2 = torch.full((rows,), -7, dtype=torch.int32, device="cuda")
+        c1 = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+        c2 = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+        assert asx.lib().asx_mask_from_activation(acts[r].data_ptr(), rows, C, mask.data_ptr(), st) == 0
+        assert asx.lib().asx_compact(mask.data_ptr(), rows, k1.data_ptr(), c1.data_ptr(), scr.data_ptr(), scr.numel() * 8, st) == 0
+        assert asx.lib().asx_compact_static(mask.data_ptr(), rows, k2.data_ptr(), c2.data_ptr(), st) == 0
+        outs.append((k1, c1, k2, c2))
+    torch.cuda.synchronize()
+    for r in range(rounds):
+        want = oracle.kept_list(oracle.mask_from_activation(acts[r].float().cpu().numpy()))
+        k1, c1, k2, c2 = outs[r]
+        assert int(c1.item()) == want.size and int(c2.item()) == want.size, r
+        assert np.array_equal(k1[:want.size].cpu().numpy(), want), r
+        assert np.array_equal(k2[:want.size].cpu().numpy(), want), r

@@ -67,8 +67,5 @@ def test_detection_stack_full_size():
 
 def test_sparsity_sweep_full_size():
     rng = np.random.default_rng(5)
-    specs = wl.config(5)
-    # every sparsity level at block 1, and the other block sizes at 50 % and 90 %
-    chosen = [s for s in specs if s.block == 1 or s.sparsity_pct in (50, 90)]
-    for spec in chosen:
+    for spec in wl.config(5):          # all 18 (sparsity, block) combinations
         _check_layer(spec, rng)

@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2309_06626_b200 as asx
 from paper_2309_06626_b200.binding import COMPACT_STATIC_MAX_ROWS
 
@@ -50,6 +51,7 @@ def test_static_compaction_matches_ordinary_entry_point_twice_in_a_row():
         got_kept, got_count = _static(md)
         assert got_count == ref_count == int(m.sum())
         assert np.array_equal(got_kept, ref_kept)
+        assert np.array_equal(got_kept, oracle.kept_list(m))          # and both equal the definition
 
 
 def test_static_compaction_rejects_sizes_beyond_its_scratch():
@@ -61,3 +63,33 @@ def test_static_compaction_rejects_sizes_beyond_its_scratch():
     assert rc == 2                                   # ASX_ERR_UNSUPPORTED, nothing launched
     assert asx.lib().asx_compact_static(small.data_ptr(), -1, out.data_ptr(), out.data_ptr(), st) == 1
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("rows", [0, 1, 16384, 16385, COMPACT_STATIC_MAX_ROWS])
+def test_static_compaction_sizes_at_the_edges_of_its_two_forms(rows):
+    """No rows, one row, the largest mask the one-block form takes, the smallest the three passes take,
+    and the largest the built-in scratch holds (every word of it in use)."""
+    rng = np.random.default_rng(rows + 3)
+    m = (rng.random(rows) < 0.37).astype(np.uint8)
+    md = torch.from_numpy(m).cuda() if rows else torch.zeros(0, dtype=torch.uint8, device="cuda")
+    got_kept, got_count = _static(md)
+    assert got_count == int(m.sum())
+    assert np.array_equal(got_kept, oracle.kept_list(m))
+
+
+@pytest.mark.parametrize("rows", [12_000, 1_600_000])
+def test_two_static_calls_without_a_synchronisation_between_them(rows):
+    """Two calls on one stream, different masks, no host synchronisation in between: the second starts
+    while the first may still be running and finds its words in the shared scratch."""
+    rng = np.random.default_rng(rows)
+    ma, mb = (rng.random(rows) < 0.6).astype(np.uint8), (rng.random(rows) < 0.2).astype(np.uint8)
+    da, db = torch.from_numpy(ma).cuda(), torch.from_numpy(mb).cuda()
+    ka, kb = (torch.full((rows,), -7, dtype=torch.int32, device="cuda") for _ in range(2))
+    ca, cb = (torch.full((1,), -7, dtype=torch.int32, device="cuda") for _ in range(2))
+    st = int(torch.cuda.current_stream().cuda_stream)
+    assert asx.lib().asx_compact_static(da.data_ptr(), rows, ka.data_ptr(), ca.data_ptr(), st) == 0
+    assert asx.lib().asx_compact_static(db.data_ptr(), rows, kb.data_ptr(), cb.data_ptr(), st) == 0
+    torch.cuda.synchronize()
+    for m, k, c in ((ma, ka, ca), (mb, kb, cb)):
+        n = int(c.item())
+        assert n == int(m.sum()) and np.array_equal(k[:n].cpu().numpy(), oracle.kept_list(m))
