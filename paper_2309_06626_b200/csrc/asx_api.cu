@@ -54,7 +54,7 @@ struct asx_layer {
     // window-patch form: the row tiles cut from the host's mask, cached per geometry and buffer size
     uint64_t tiles_epoch = ~0ull;
     int tiles_Nb = 0, tiles_H = 0, tiles_W = 0, tiles_cap = 0;
-    std::vector<int32_t> host_tiles;   // pairs: first kept lowered row, rows
+    std::vector<int32_t> host_tiles;   // per tile: first kept lowered row, rows, first padded input row of its patch, patch rows
     int64_t tiles_rows = 0;            // kept lowered rows they cover
     void* d_tiles = nullptr;
     size_t d_tiles_bytes = 0;
@@ -152,7 +152,8 @@ void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]
 
 // Window-patch form: cut the kept lowered rows (ascending in image and output row) into tiles of at
 // most 128 consecutive rows whose windows span at most `cap` zero-padded input rows.  Pure index
-// bookkeeping on the mask the host holds; returns the kept lowered rows, or -1 without memory.
+// bookkeeping on the mask the host holds; four ints per tile (first kept lowered row, rows, first
+// padded input row of the patch, patch rows); returns the kept lowered rows, or -1 without memory.
 int64_t cut_row_tiles(const std::vector<uint8_t>& mask, int Nb, int P, int Wo, int Hp, int kh, int cap, std::vector<int32_t>* tiles)
 {
     std::vector<int32_t> kept;
@@ -174,6 +175,8 @@ int64_t cut_row_tiles(const std::vector<uint8_t>& mask, int Nb, int P, int Wo, i
             while (n < 128 && r0 + n < Mk && padded_row(r0 + n) - first + kh <= cap) ++n;
             tiles->push_back((int32_t)r0);
             tiles->push_back((int32_t)n);
+            tiles->push_back((int32_t)first);                                     // first padded input row of the patch
+            tiles->push_back((int32_t)(padded_row(r0 + n - 1) - first + kh));     // its rows
             r0 += n;
         }
         return Mk;
@@ -642,7 +645,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
             }
         }
         if (L->tiles_rows > 0 && L->tiles_rows == est_rows) {
-            plan_patch_cost(g, L->num_sms, (long long)(L->host_tiles.size() / 2), &pplan);
+            plan_patch_cost(g, L->num_sms, (long long)(L->host_tiles.size() / 4), &pplan);
             use_patch = pplan.est_cost_us <= plan.est_cost_us || (flags & ASX_IMPL_WINDOW_PATCH);
         }
     }
@@ -696,7 +699,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         }
         L->last_form = ASX_FORM_WINDOW_PATCH;
         return from_cuda(launch_patch(g, pplan, L->tmap, L->tmap_x4, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status, L->num_sms,
-                                      fuse_compact ? 1 : 0, L->host_kept, L->residual, L->d_tiles, (int)(L->host_tiles.size() / 2), L->tiles_rows,
+                                      fuse_compact ? 1 : 0, L->host_kept, L->residual, L->d_tiles, (int)(L->host_tiles.size() / 4), L->tiles_rows,
                                       L->wait_limit_kcycles, st));
     }
     if (plan.vec == 2) {

@@ -76,7 +76,8 @@ __device__ __forceinline__ bool warp_wait_bar(uint32_t bar, uint32_t parity, vol
 // (16 bytes per thread, popcount, shuffle scan within the warps, warp totals through shared
 // memory) and writes the ascending kept positions as 16-bit values into its own shared memory
 // (every block writing the list to the same global addresses serialises in L2 and cost 10-20 us;
-// block 0 alone copies it out).  Returns the count.
+// block 0 alone copies it out).  Returns the count.  The first `nthreads` threads of the block take part
+// (a multiple of 32; they meet on hardware barrier `barrier_id`), the others may do something else.
 // Bit q of the result: byte q of the 16 mask bytes in v is non-zero.
 __device__ __forceinline__ unsigned nonzero_bytes16(const uint4& v)
 {
@@ -103,7 +104,7 @@ __device__ __forceinline__ unsigned mask_flags16(const uint8_t* __restrict__ mas
 // `early` holds mask bytes 16 tid .. 16 tid + 15 when `early_ok` (the caller read them before the
 // kernel's set-up so that the latency of the read is hidden behind it).
 __device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, int rows, const uint4& early, bool early_ok,
-                                             unsigned short* kept_s, int* scan_total, int nthreads)
+                                             unsigned short* kept_s, int* scan_total, int nthreads, int barrier_id = 0)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = nthreads >> 5;
     int running = 0;
@@ -123,7 +124,7 @@ __device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, i
             }
         }
         if (lane == 31) scan_total[warp] = incl;
-        __syncthreads();
+        asm volatile("bar.sync %0, %1;" ::"r"(barrier_id), "r"(nthreads) : "memory");
         if (wactive) {
             // scan of the (at most 27) warp totals with shuffles
             const int wt = lane < nwarps ? scan_total[lane] : 0;
@@ -144,7 +145,7 @@ __device__ __forceinline__ int block_compact(const uint8_t* __restrict__ mask, i
             }
             if (tid == 0) scan_total[31] = running + total;     // slot 31 is no warp's total (27 warps)
         }
-        __syncthreads();
+        asm volatile("bar.sync %0, %1;" ::"r"(barrier_id), "r"(nthreads) : "memory");
         running = scan_total[31];
     }
     return running;

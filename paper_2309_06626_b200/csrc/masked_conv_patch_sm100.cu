@@ -46,9 +46,13 @@ constexpr int MAX_B_STAGES = 8;
 constexpr int MAX_A_STAGES = 12;
 constexpr int TAP_COLS = 32;            // 64 bf16 per row = 32 columns of tensor memory per filter tap
 constexpr int FULL_RING = 24;           // 'stage full' barriers: a multiple of every A and filter ring depth in use (2, 3, 4)
-constexpr int W_FILTER = 0, W_MMA = 1, W_EPI0 = 2, NUM_EPI_WARPS = 4, W_PATCH = 6, W_INFO = 7, W_FILL0 = 8,
-              NUM_FILL_WARPS = 16, W_ZERO0 = W_FILL0 + NUM_FILL_WARPS, NUM_ZERO_WARPS = 4;
-constexpr int NUM_THREADS = 32 * (W_ZERO0 + NUM_ZERO_WARPS);
+// Warp roles.  The two loader warps come last: they take no part in the mask compaction and the row
+// decoding (threads 0 .. WORK_THREADS-1 do, meeting on hardware barrier 2) but start fetching filter
+// slabs and input patches as soon as the barriers exist, from the tile table the host cut.
+constexpr int W_MMA = 0, W_INFO = 1, W_EPI0 = 2, NUM_EPI_WARPS = 4, W_ZERO_A = 6, W_FILL0 = 8, NUM_FILL_WARPS = 16,
+              W_ZERO_B = 24, NUM_ZERO_WARPS = 4, W_FILTER = 26, W_PATCH = 27;
+constexpr int WORK_THREADS = 32 * W_FILTER;
+constexpr int NUM_THREADS = 32 * (W_PATCH + 1);
 static_assert(NUM_THREADS / 32 < 32, "the fused compaction keeps its running count in slot 31 of the warp totals");
 static_assert((W_FILL0 & 3) == 0 && (NUM_FILL_WARPS & 3) == 0, "fill warps come in groups of four lane quarters");
 
@@ -73,16 +77,15 @@ struct PatchArgs {
     int32_t* kept_out;
     int32_t* count_out;
     const __nv_bfloat16* residual;
-    const int2* tiles;  // per row tile: first kept lowered row, number of rows (1..128); cut by the host from the mask
+    const int4* tiles;  // per row tile: first kept lowered row, number of rows (1..128), first padded input row of
+                        // its patch, patch rows; cut by the host from the mask
     int n_mtiles;       // row tiles
     int Mk_host;        // kept lowered rows the tiles cover; must equal what the device counts
     int wait_limit_kcycles;
 };
 
 struct alignas(16) PShared {          // lives after the patch buffers and the filter stages
-    int rowpix[INFO_RING][BM];        // per tile row: (padded input row of the window's top) * Wp8 + ox, or -1
-    int tile_lo[INFO_RING];           // first and last padded input row of the tile's patch
-    int tile_hi[INFO_RING];
+    int rowpix[INFO_RING][BM];        // per tile row: pixel index of the window's corner within the tile's patch, or -1
     float bias[2][128];
     unsigned long long info_full[INFO_RING];
     unsigned long long info_empty[INFO_RING];
@@ -130,17 +133,24 @@ __device__ __forceinline__ PItem pitem_of(int t, const PatchArgs& a)
     return it;
 }
 
-// Row coordinates of one tile row into ring slot jj; the threads that decode the tile's first and
-// last row also record the patch's row range.
+// Row coordinates of one tile row into ring slot jj, relative to the tile's patch.
 __device__ __forceinline__ void decode_row(PShared* sh, int jj, int rr, int m_tile, int Mk, const FastDiv& fdcnt,
                                            const ConvGeom& g, const PatchArgs& a, const KeptList& kept)
 {
-    const int2 tl = __ldg(a.tiles + m_tile);            // written by a stream-ordered copy, never by a kernel
+    const int4 tl = __ldg(a.tiles + m_tile);            // written by a stream-ordered copy, never by a kernel
     int prow;
     const int px = row_pixel_of(rr < tl.y ? tl.x + rr : Mk, Mk, fdcnt, g, a, kept, &prow);
-    sh->rowpix[jj][rr] = px;
-    if (rr == 0) sh->tile_lo[jj] = prow < 0 ? 0 : prow;
-    if (rr == tl.y - 1) sh->tile_hi[jj] = prow < 0 ? 0 : prow + g.kh - 1;
+    // relative to the patch's first pixel; a row whose window the host's patch range does not cover
+    // (the table was cut for another mask) is flagged and reads pixel 0
+    int rel = -1;
+    if (px >= 0) {
+        rel = px - tl.z * a.Wp8;
+        if (prow < tl.z || prow + g.kh > tl.z + tl.w || tl.w > a.cap_rows) {
+            atomicOr(a.dev_status, DEV_BAD_INDEX);
+            rel = -1;
+        }
+    }
+    sh->rowpix[jj][rr] = rel;
 }
 
 template <bool RESIDUAL, bool SILU>
@@ -170,7 +180,7 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
     volatile WaitCtl* ctl = &sh->ctl;
 
     uint4 early_mask = make_uint4(0, 0, 0, 0);
-    const bool early_ok = a.fuse_compact && tid * 16 + 16 <= g.rows && (reinterpret_cast<uintptr_t>(a.mask) & 15) == 0;
+    const bool early_ok = a.fuse_compact && tid < WORK_THREADS && tid * 16 + 16 <= g.rows && (reinterpret_cast<uintptr_t>(a.mask) & 15) == 0;
     if (early_ok) early_mask = ptx::ld_global_v4_keep_in_l2(a.mask + tid * 16);
 
     // barrier initialisation, one barrier per thread (a single thread took about 1500 clocks over them)
@@ -184,7 +194,7 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
             else if ((i -= FULL_RING) < MAX_B_STAGES) { bar = &sh->b_empty[i]; count = 1; }
             else if ((i -= MAX_B_STAGES) < MAX_A_STAGES) { bar = &sh->a_empty[i]; count = 1; }
             else if ((i -= MAX_A_STAGES) < INFO_RING) { bar = &sh->info_full[i]; count = 1; }
-            else if ((i -= INFO_RING) < INFO_RING) { bar = &sh->info_empty[i]; count = NUM_FILL_WARPS + 1; }   // the fill warps and the patch thread
+            else if ((i -= INFO_RING) < INFO_RING) { bar = &sh->info_empty[i]; count = NUM_FILL_WARPS; }
             else if ((i -= INFO_RING) < 2) { bar = &sh->p_full[i]; count = 1; }
             else if ((i -= 2) < 2) { bar = &sh->p_empty[i]; count = NUM_FILL_WARPS; }
             else if ((i -= 2) < 2) { bar = &sh->acc_full[i]; count = 1; }
@@ -209,20 +219,90 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
     const uint32_t tmem_base = sh->tmem_base;
     const uint32_t a_col0 = (uint32_t)(2 * BN);                      // the A stages follow the two accumulators
 
+    const int host_tiles = a.n_mtiles * a.n_tiles;      // what the host's tile table says; the workers check it against the mask
+    if (warp >= W_FILTER) {
+        // ================================================================== loader warps
+        // They need neither the kept-row list nor the row coordinates: the tile table gives each tile's
+        // patch range, so the first filter slabs and the first patches are on their way while the other
+        // warps still compact the mask and decode rows.  Each loader thread waits for the preceding
+        // kernel by itself before its first load.
+        if (lane == 0) {
+            ptx::grid_dependency_wait();
+            bool ok = true;
+            if (warp == W_FILTER) {
+                // ---------------------------------------------------------- filter slabs by TMA
+                // Stages run slice by slice (all taps of channels 64 s .. 64 s + 63, then the next slice),
+                // so that one slice of the patch is in use at a time; in w[C_out][kh][kw][C_in] the slab
+                // of (tap, slice) starts at K index tap * C_in + 64 * slice.
+                int s = 0, fi = 0;
+                uint32_t ph = 0;
+                for (int t = blockIdx.x; t < host_tiles && ok; t += gridDim.x) {
+                    const int n_tile = pitem_of(t, a).n_tile;
+                    for (int sl = 0; sl < a.slices && ok; ++sl)
+                        for (int tap0 = 0; tap0 < taps; tap0 += G) {
+                            const int gc = taps - tap0 < G ? taps - tap0 : G;
+                            if (!wait_bar<40>(ptx::smem_u32(&sh->b_empty[s]), ph ^ 1u, ctl, a.dev_status)) { ok = false; break; }
+                            const uint32_t full = ptx::smem_u32(&sh->full[fi]);
+                            ptx::mbar_arrive_expect_tx(full, (uint32_t)gc * b_tap_bytes);
+                            for (int i = 0; i < gc; ++i)
+                                ptx::tma_load_2d(b_base + (uint32_t)s * b_stage_bytes + (uint32_t)i * b_tap_bytes, &tmap_w, full,
+                                                 (tap0 + i) * g.C_in + sl * 64, n_tile * BN);
+                            if (++s == BS) { s = 0; ph ^= 1u; }
+                            if (++fi == FULL_RING) fi = 0;
+                        }
+                }
+            } else {
+                // ---------------------------------------------------------- input patches by TMA
+                // Per tile and slice: the padded input rows of the tile's patch, one box of Wp pixels x 64
+                // channels each, starting Wp8 pixels apart in the buffer (every box 1024-byte aligned, so
+                // the 128-byte swizzle phase of a pixel is its index within the buffer modulo 8).
+                uint32_t use = 0;
+                for (int t = blockIdx.x; t < host_tiles && ok; t += gridDim.x) {
+                    const int4 tl = __ldg(a.tiles + pitem_of(t, a).m_tile);
+                    int nrows = tl.w;
+                    if (nrows > a.cap_rows || nrows < 1) {                 // cannot happen when the host planned from this mask
+                        atomicOr(a.dev_status, DEV_BAD_INDEX);
+                        nrows = nrows < 1 ? 1 : a.cap_rows;
+                    }
+                    const int n_lo = (int)fd_div((uint32_t)tl.z, a.fdHp);
+                    for (int sl = 0; sl < a.slices; ++sl, ++use) {
+                        const uint32_t b = use & 1u;
+                        if (!wait_bar<40>(ptx::smem_u32(&sh->p_empty[b]), ((use >> 1) & 1u) ^ 1u, ctl, a.dev_status)) { ok = false; break; }
+                        const uint32_t full = ptx::smem_u32(&sh->p_full[b]);
+                        ptx::mbar_arrive_expect_tx(full, (uint32_t)nrows * (uint32_t)a.Wp * 128u);
+                        int n = n_lo, yy = tl.z - n_lo * a.Hp;             // padded row yy of image n
+                        uint32_t dst = smem_base + b * patch_bytes;
+                        for (int i = 0; i < nrows; ++i) {
+                            ptx::tma_load_4d(dst, &tmap_x, full, sl * 64, -g.pad_w, yy - g.pad, n);
+                            dst += row_bytes;
+                            if (++yy == a.Hp) { yy = 0; ++n; }
+                        }
+                    }
+                }
+            }
+            if (!ok) {   // let loads already issued land before the block's shared memory goes away
+                for (int i = 0; i < 64; ++i) __nanosleep(1000);
+            }
+        }
+    } else {
+    // ====================================================================== worker warps
     int cnt = 0;
     KeptList kept_list{a.kept, nullptr};
     unsigned short* kept_s = reinterpret_cast<unsigned short*>(sh + 1);
     if (a.fuse_compact) {
-        cnt = block_compact(a.mask, g.rows, early_mask, early_ok, kept_s, sh->scan_total, NUM_THREADS);
+        cnt = block_compact(a.mask, g.rows, early_mask, early_ok, kept_s, sh->scan_total, WORK_THREADS, 2);
         kept_list.s = kept_s;
     } else {
         ptx::grid_dependency_wait();
         cnt = __ldcg(a.count);
     }
     const int Mk = (g.rows == g.P) ? g.Nb * cnt : cnt;
-    int total_tiles = a.n_mtiles * a.n_tiles;
+    int total_tiles = host_tiles;
     if (Mk != a.Mk_host) {                     // the tiles were cut for another mask: nothing can be computed
-        if (tid == 0) atomicOr(a.dev_status, DEV_BAD_INDEX);
+        if (tid == 0) {
+            atomicOr(a.dev_status, DEV_BAD_INDEX);
+            sh->ctl.abort = 1;                 // the loader warps leave their waits
+        }
         total_tiles = 0;
     }
     FastDiv fdcnt = a.fdcnt_host;
@@ -230,89 +310,23 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
 
     // Row coordinates of this block's first INFO_RING tiles, one row per thread.
     {
-        for (int idx = tid; idx < INFO_RING * BM; idx += NUM_THREADS) {
+        for (int idx = tid; idx < INFO_RING * BM; idx += WORK_THREADS) {
             const int jj = idx / BM, rr = idx - jj * BM;
             const long long t = blockIdx.x + (long long)jj * gridDim.x;
             if (t < total_tiles) decode_row(sh, jj, rr, pitem_of((int)t, a).m_tile, Mk, fdcnt, g, a, kept_list);
         }
-        __syncthreads();
+        asm volatile("bar.sync 2, %0;" ::"n"(WORK_THREADS) : "memory");
         if (tid < INFO_RING && blockIdx.x + (long long)tid * gridDim.x < total_tiles) ptx::mbar_arrive(ptx::smem_u32(&sh->info_full[tid]));
     }
     if (a.fuse_compact) {
         ptx::grid_dependency_wait();
         if (blockIdx.x == 0) {      // the list in global memory, for asx_get_kept and later runs
-            for (int i = tid; i < cnt; i += NUM_THREADS) a.kept_out[i] = (int32_t)kept_s[i];
+            for (int i = tid; i < cnt; i += WORK_THREADS) a.kept_out[i] = (int32_t)kept_s[i];
             if (tid == 0) *a.count_out = cnt;
         }
     }
 
-    if (warp == W_FILTER) {
-        // ------------------------------------------------------------------ filter slabs by TMA
-        // k-blocks run slice by slice (all taps of channels 64 s .. 64 s + 63, then the next slice),
-        // so that one slice of the patch is in use at a time; in w[C_out][kh][kw][C_in] the slab of
-        // (tap, slice) starts at K index tap * C_in + 64 * slice.
-        if (lane == 0) {
-            int s = 0, fi = 0;
-            uint32_t ph = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const int n_tile = pitem_of(t, a).n_tile;
-                for (int sl = 0; sl < a.slices && ok; ++sl)
-                    for (int tap0 = 0; tap0 < taps; tap0 += G) {
-                        const int gc = taps - tap0 < G ? taps - tap0 : G;
-                        if (!wait_bar<40>(ptx::smem_u32(&sh->b_empty[s]), ph ^ 1u, ctl, a.dev_status)) { ok = false; break; }
-                        const uint32_t full = ptx::smem_u32(&sh->full[fi]);
-                        ptx::mbar_arrive_expect_tx(full, (uint32_t)gc * b_tap_bytes);
-                        for (int i = 0; i < gc; ++i)
-                            ptx::tma_load_2d(b_base + (uint32_t)s * b_stage_bytes + (uint32_t)i * b_tap_bytes, &tmap_w, full,
-                                             (tap0 + i) * g.C_in + sl * 64, n_tile * BN);
-                        if (++s == BS) { s = 0; ph ^= 1u; }
-                        if (++fi == FULL_RING) fi = 0;
-                    }
-            }
-            if (!ok) {   // let loads already issued land before the block's shared memory goes away
-                for (int i = 0; i < 64; ++i) __nanosleep(1000);
-            }
-        }
-    } else if (warp == W_PATCH) {
-        // ------------------------------------------------------------------ input patches by TMA
-        // Per tile and slice: padded input rows tile_lo .. tile_hi, one box of Wp pixels x 64
-        // channels each, starting Wp8 pixels apart in the buffer (every box 1024-byte aligned, so the
-        // 128-byte swizzle phase of a pixel is its index within the buffer modulo 8).
-        if (lane == 0) {
-            uint32_t use = 0;
-            int j = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++j) {
-                const int r = j & (INFO_RING - 1);
-                if (!wait_bar<100>(ptx::smem_u32(&sh->info_full[r]), (uint32_t)(j / INFO_RING) & 1u, ctl, a.dev_status)) break;
-                const int lo = sh->tile_lo[r];
-                int nrows = sh->tile_hi[r] - lo + 1;
-                ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));
-                if (nrows > a.cap_rows || nrows < 1) {                 // cannot happen when the host planned from this mask
-                    atomicOr(a.dev_status, DEV_BAD_INDEX);
-                    nrows = nrows < 1 ? 1 : a.cap_rows;
-                }
-                const int n_lo = (int)fd_div((uint32_t)lo, a.fdHp);
-                for (int sl = 0; sl < a.slices; ++sl, ++use) {
-                    const uint32_t b = use & 1u;
-                    if (!wait_bar<40>(ptx::smem_u32(&sh->p_empty[b]), ((use >> 1) & 1u) ^ 1u, ctl, a.dev_status)) { ok = false; break; }
-                    const uint32_t full = ptx::smem_u32(&sh->p_full[b]);
-                    ptx::mbar_arrive_expect_tx(full, (uint32_t)nrows * (uint32_t)a.Wp * 128u);
-                    int n = n_lo, yy = lo - n_lo * a.Hp;               // padded row yy of image n
-                    uint32_t dst = smem_base + b * patch_bytes;
-                    for (int i = 0; i < nrows; ++i) {
-                        ptx::tma_load_4d(dst, &tmap_x, full, sl * 64, -g.pad_w, yy - g.pad, n);
-                        dst += row_bytes;
-                        if (++yy == a.Hp) { yy = 0; ++n; }
-                    }
-                }
-            }
-            if (!ok) {
-                for (int i = 0; i < 64; ++i) __nanosleep(1000);
-            }
-        }
-    } else if (warp == W_INFO) {
+    if (warp == W_INFO) {
         // ------------------------------------------------------------------ row coordinates
         int j = INFO_RING;                        // the first INFO_RING tiles were decoded by the whole block
         for (long long t = blockIdx.x + (long long)INFO_RING * gridDim.x; t < total_tiles; t += gridDim.x, ++j) {
@@ -381,7 +395,7 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
             const int n0 = item.n_tile * BN;
             const int buf = ti & 1;
             const uint32_t use = (uint32_t)(ti >> 1) & 1u;
-            const int2 tl = __ldg(a.tiles + item.m_tile);
+            const int4 tl = __ldg(a.tiles + item.m_tile);
             const int rk = tl.x + q * 32 + lane;
             const bool valid = q * 32 + lane < tl.y;
             const long long yoff = valid ? (long long)out_row_of(rk, fdcnt, g, kept_list) * N : 0;
@@ -442,9 +456,9 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[buf]));
         }
-    } else if (warp >= W_ZERO0) {
+    } else if (warp == W_ZERO_A || warp == W_ZERO_A + 1 || warp == W_ZERO_B || warp == W_ZERO_B + 1) {
         // ------------------------------------------------------------------ zeros for dropped rows
-        zero_fill_dropped_rows<false, NUM_ZERO_WARPS * 32>(a.y, a.mask, g, 1, (warp - W_ZERO0) * 32 + lane);
+        zero_fill_dropped_rows<false, NUM_ZERO_WARPS * 32>(a.y, a.mask, g, 1, ((warp >= W_ZERO_B ? warp - W_ZERO_B + 2 : warp - W_ZERO_A) * 32 + lane));
     } else {
         // ------------------------------------------------------------------ A operand: patch -> tensor memory
         // Warp (quarter q, group grp) owns tile rows 32 q .. 32 q + 31 (tensor-memory lanes a warp can
@@ -464,10 +478,9 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
             const int r = j & (INFO_RING - 1);
             if (!warp_wait_bar<100>(ptx::smem_u32(&sh->info_full[r]), (uint32_t)(j / INFO_RING) & 1u, ctl, a.dev_status)) break;
             const int px = sh->rowpix[r][q * 32 + lane];
-            const int lo = sh->tile_lo[r];
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_empty[r]));        // the ring slot is in registers now
-            int base = px >= 0 ? px - lo * a.Wp8 : 0;                                  // rows past the end read pixel 0; their results are never stored
+            int base = px >= 0 ? px : 0;                                           // rows past the end read pixel 0; their results are never stored
             base = base < 0 ? 0 : (base > max_base ? max_base : base);
             for (int sl = 0; sl < a.slices && ok; ++sl, ++use) {
                 const uint32_t b = use & 1u;
@@ -509,6 +522,8 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
             }
         }
     }
+
+    }   // worker warps
 
     ptx::tc_fence_before_sync();
     __syncthreads();
@@ -611,7 +626,7 @@ cudaError_t launch_patch(const ConvGeom& g, const PatchPlan& plan, const CUtenso
     a.count_out = const_cast<int32_t*>(count);
     a.residual = static_cast<const __nv_bfloat16*>(residual);
     a.wait_limit_kcycles = wait_limit_kcycles > 0 ? wait_limit_kcycles : WAIT_LIMIT_KCYCLES_DEFAULT;
-    a.tiles = static_cast<const int2*>(tiles);
+    a.tiles = static_cast<const int4*>(tiles);
     a.n_mtiles = n_mtiles;
     a.Mk_host = (int)kept_rows;
 
