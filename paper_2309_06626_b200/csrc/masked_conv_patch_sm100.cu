@@ -68,6 +68,7 @@ struct PatchArgs {
     const int32_t* count;
     int* dev_status;
     int relu;
+    int st32;           // 32-byte epilogue stores: C_out % 16 == 0, BN % 16 == 0 and y 32-byte aligned
     int BN, n_tiles, b_stages, a_stages;
     int cap_rows;       // padded input rows one patch buffer holds
     int Hp, Wp, Wp8;    // padded input height and width; Wp rounded up to a multiple of 8 (row pitch in pixels)
@@ -423,6 +424,8 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
                 }
                 ptx::tmem_ld_wait();
                 if (valid) {
+                    uint4 ov[4];
+                    int nh = 0;
 #pragma unroll
                     for (int h = 0; h < 4; ++h) {
                         const int colh = col0 + 8 * h;
@@ -443,12 +446,25 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
 #pragma unroll
                             for (int j = 0; j < 8; ++j) v[j] = fmaxf(v[j], 0.f);
                         }
-                        uint4 o;
-                        o.x = pack_bf16(v[0], v[1]);
-                        o.y = pack_bf16(v[2], v[3]);
-                        o.z = pack_bf16(v[4], v[5]);
-                        o.w = pack_bf16(v[6], v[7]);
-                        *reinterpret_cast<uint4*>(y2 + yoff + colh) = o;
+                        ov[h].x = pack_bf16(v[0], v[1]);
+                        ov[h].y = pack_bf16(v[2], v[3]);
+                        ov[h].z = pack_bf16(v[4], v[5]);
+                        ov[h].w = pack_bf16(v[6], v[7]);
+                        nh = h + 1;
+                    }
+                    // a kept row's neighbours in memory are mostly dropped rows, so this thread's stores share
+                    // their sectors with no other thread: whole 32-byte sectors where the layout allows
+                    unsigned short* dst = y2 + yoff + col0;
+                    if (a.st32) {
+#pragma unroll
+                        for (int h = 0; h < 4; h += 2) {
+                            if (h + 1 < nh) ptx::st_global_v8(dst + 8 * h, ov[h], ov[h + 1]);
+                            else if (h < nh) *reinterpret_cast<uint4*>(dst + 8 * h) = ov[h];
+                        }
+                    } else {
+#pragma unroll
+                        for (int h = 0; h < 4; ++h)
+                            if (h < nh) *reinterpret_cast<uint4*>(dst + 8 * h) = ov[h];
                     }
                 }
             }
@@ -611,6 +627,7 @@ cudaError_t launch_patch(const ConvGeom& g, const PatchPlan& plan, const CUtenso
     a.count = count;
     a.dev_status = dev_status;
     a.relu = relu == 1 ? 1 : 0;
+    a.st32 = (g.C_out % 16 == 0 && (reinterpret_cast<uintptr_t>(y) & 31) == 0) ? 1 : 0;
     a.BN = plan.BN;
     a.n_tiles = plan.n_tiles;
     a.b_stages = plan.b_stages;

@@ -116,6 +116,16 @@ __device__ __forceinline__ void ld_shared_v4(uint32_t src, uint32_t& a, uint32_t
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(src));
 }
 
+// 32-byte global store (one whole sector from one thread; the address must be 32-byte aligned).  A
+// 16-byte store from a thread whose neighbours write other lines occupies a full sector's slot on
+// the way to L2, so two of them cost twice the bandwidth of this.
+__device__ __forceinline__ void st_global_v8(void* p, const uint4& a, const uint4& b)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w),
+                 "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
+                 : "memory");
+}
+
 // 16-byte global load that asks L2 to keep the line when it has to evict (for small read-only
 // data that every launch reads first, while the launches in between stream through L2).
 __device__ __forceinline__ uint4 ld_global_v4_keep_in_l2(const void* p)
