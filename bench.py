@@ -35,14 +35,13 @@ RECOMPACT_FLAG = 2          # ASX_RECOMPACT: every step rebuilds the kept-row li
 L2_BYTES = 126 * 1024 * 1024
 
 
-# DRAM traffic of the dominant kernel from one ncu capture of the default workload (ResNet-18 stack,
-# batch 64): dram__bytes_read.sum + dram__bytes_write.sum averaged over the 20 fused-kernel launches
-# of a step (12.18 MB read + 2.37 MB written; ncu flushes the caches before every captured launch,
-# so reads are cold-cache and most of a launch's output is still in L2 when its counters stop).
-# The figure belongs to the kernel sources whose digest is recorded with it; with any other sources
-# the bench reports null.
-NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 14.54e6,
-               "csrc_sha256": "fbfd4091dd51ba734e7f9d2fe1af3a30db7a829569e92f869aac216077f4f393"}
+# DRAM traffic of the fused kernels from one ncu capture of the default workload (ResNet-18 stack, batch 64):
+# dram__bytes_read.sum + dram__bytes_write.sum averaged over the 20 fused-kernel launches of a step
+# (12.77 MB read + 2.41 MB written; ncu flushes the caches before every captured launch, so reads are
+# cold-cache and most of a launch's output is still in L2 when its counters stop).  The figure belongs to
+# the kernel sources whose digest is recorded with it; with any other sources the bench reports null.
+NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 15.18e6,
+               "csrc_sha256": "b6fbd25dddef01f1327a1001a6399723ef4734363fa01a6ffbdf82fcd5b9e3e0"}
 
 
 def csrc_digest() -> str:
