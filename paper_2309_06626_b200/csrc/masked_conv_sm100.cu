@@ -62,6 +62,7 @@ struct FastArgs {
     int relu;
     int BN, n_tiles, stages, tmem_cols;
     int vec_out;        // C_out % 8 == 0 and y 16-byte aligned: 16-byte stores
+    int st32;           // bf16, C_out % 16 == 0, y 32-byte aligned and the layer is paced by its stores: 32-byte epilogue stores
     int fuse_compact;   // rebuild the kept-row list from the mask inside this kernel (small masks)
     int32_t* kept_out;  // where the fused compaction writes the list and its count
     int32_t* count_out;
@@ -496,6 +497,7 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                 }
                 ptx::tmem_ld_wait();
                 if (valid) {
+                    uint4 hold = make_uint4(0, 0, 0, 0);
 #pragma unroll
                     for (int h = 0; h < 4; ++h) {
                         const int colh = col0 + 8 * h;
@@ -532,7 +534,12 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                             o.y = pack_bf16(v[2], v[3]);
                             o.z = pack_bf16(v[4], v[5]);
                             o.w = pack_bf16(v[6], v[7]);
-                            *reinterpret_cast<uint4*>(y2 + yoff + colh) = o;
+                            if (a.st32) {              // C_out % 16 == 0: chunks come in pairs, one whole sector per store
+                                if (h & 1) ptx::st_global_v8(y2 + yoff + colh - 8, hold, o);
+                                else hold = o;
+                            } else {
+                                *reinterpret_cast<uint4*>(y2 + yoff + colh) = o;
+                            }
                         } else {
 #pragma unroll
                             for (int j = 0; j < 8; ++j)
@@ -918,6 +925,10 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
     while (cols < 2 * plan.BN) cols <<= 1;
     a.tmem_cols = cols;
     a.vec_out = (g.C_out % (f32 ? 4 : 8) == 0 && (reinterpret_cast<uintptr_t>(y) & 15) == 0) ? 1 : 0;
+    // Whole-sector stores pay where the epilogue's stores pace the kernel: few k-blocks per tile (the network's
+    // first layers, 1x1 convolutions) and rows that are written without a residual read in between.
+    a.st32 = (!f32 && a.vec_out && g.C_out % 16 == 0 && plan.BN % 16 == 0 && (reinterpret_cast<uintptr_t>(y) & 31) == 0 &&
+              plan.ksplit == 1 && out_compact == 0) ? 1 : 0;
 
     long long tiles = ((long long)g.M + BM - 1) / BM * plan.n_tiles * plan.ksplit;
     int grid = (int)(tiles < num_sms ? tiles : num_sms);
