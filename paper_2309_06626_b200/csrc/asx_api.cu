@@ -622,10 +622,10 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     if (!plan_fast(g, L->num_sms, est_rows, fuse_compact ? (int)L->rows : 0, allow_split, ES, &plan)) return ASX_ERR_UNSUPPORTED;
     // Stride-1 layers with several filter taps and whole 64-channel slices take the window-patch form
     // when the host knows the mask, every tile's windows fit the patch buffers and the planner's
-    // estimate favours it; compact tensors and fp32 storage stay with the row gather.
+    // estimate favours it; compact inputs and fp32 storage stay with the row gather.
     PatchPlan pplan;
     bool use_patch = false;
-    if (!f32 && !in_compact && !out_compact && !(flags & ASX_IMPL_ROW_GATHER) && !L->host_mask.empty() &&
+    if (!f32 && !in_compact && !(flags & ASX_IMPL_ROW_GATHER) && !L->host_mask.empty() &&
         (reinterpret_cast<uintptr_t>(y) & 15) == 0 && plan_patch(g, fuse_compact ? (int)L->rows : 0, &pplan)) {
         if (L->tiles_epoch != L->mask_epoch || L->tiles_Nb != Nb || L->tiles_H != H || L->tiles_W != W || L->tiles_cap != pplan.cap_rows) {
             L->tiles_rows = cut_row_tiles(L->host_mask, Nb, g.P, g.Wo, pplan.Hp, g.kh, pplan.cap_rows, &L->host_tiles);
@@ -700,7 +700,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         L->last_form = ASX_FORM_WINDOW_PATCH;
         return from_cuda(launch_patch(g, pplan, L->tmap, L->tmap_x4, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status, L->num_sms,
                                       fuse_compact ? 1 : 0, L->host_kept, L->residual, L->d_tiles, (int)(L->host_tiles.size() / 4), L->tiles_rows,
-                                      L->wait_limit_kcycles, st));
+                                      out_compact ? 1 : 0, L->wait_limit_kcycles, st));
     }
     if (plan.vec == 2) {
         const int64_t pixels = in_compact ? x_rows : (int64_t)Nb * g.H * g.W;

@@ -79,7 +79,7 @@ cudaError_t launch_fast(const ConvGeom& g, const FastPlan& plan, const CUtensorM
                         int out_compact, const int32_t* in_rank, int in_kept, const void* residual, int f32, int wait_limit_kcycles,
                         cudaStream_t st);
 // ---- the window-patch form of the tensor-core path (masked_conv_patch_sm100.cu): stride-1 layers with
-// several filter taps and C_in % 64 == 0, bf16, dense input and output
+// several filter taps and C_in % 64 == 0, bf16, dense input, dense or compact output
 struct PatchPlan {
     int BN, n_tiles;
     int a_stages, b_stages;
@@ -97,8 +97,8 @@ void plan_patch_cost(const ConvGeom& g, int num_sms, long long n_mtiles, PatchPl
 cudaError_t launch_patch(const ConvGeom& g, const PatchPlan& plan, const CUtensorMap& tmap_w, const CUtensorMap& tmap_x4,
                          const float* bias, void* y, const uint8_t* mask, const int32_t* kept, const int32_t* count,
                          int relu, int* dev_status, int num_sms, int fuse_compact, long long host_kept,
-                         const void* residual, const void* tiles, int n_mtiles, long long kept_rows, int wait_limit_kcycles,
-                         cudaStream_t st);
+                         const void* residual, const void* tiles, int n_mtiles, long long kept_rows, int out_compact,
+                         int wait_limit_kcycles, cudaStream_t st);
 // src[rows][C] -> dst[rows][Cp] with zero channels added (Cp = 4 or a multiple of 8; rows*Cp % 8 == 0)
 cudaError_t launch_pad_channels(const void* src, void* dst, long long rows, int C, int Cp, cudaStream_t st);
 // filters for the pixel-pair form: w[C_out][kh][kw][C] -> w2[C_out][kh][kw2][2][4], where pair kxx,

@@ -68,6 +68,7 @@ struct PatchArgs {
     const int32_t* count;
     int* dev_status;
     int relu;
+    int out_compact;    // y holds the kept rows only, in kept order (row rk at y[rk][*]); nothing is zero-filled
     int st32;           // 32-byte epilogue stores: C_out % 16 == 0, BN % 16 == 0 and y 32-byte aligned
     int BN, n_tiles, b_stages, a_stages;
     int cap_rows;       // padded input rows one patch buffer holds
@@ -399,7 +400,7 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
             const int4 tl = __ldg(a.tiles + item.m_tile);
             const int rk = tl.x + q * 32 + lane;
             const bool valid = q * 32 + lane < tl.y;
-            const long long yoff = valid ? (long long)out_row_of(rk, fdcnt, g, kept_list) * N : 0;
+            const long long yoff = valid ? (long long)(a.out_compact ? rk : out_row_of(rk, fdcnt, g, kept_list)) * N : 0;
             {
                 float* sb = sh->bias[buf];
                 const int et = (warp - W_EPI0) * 32 + lane;
@@ -473,8 +474,8 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->acc_empty[buf]));
         }
     } else if (warp == W_ZERO_A || warp == W_ZERO_A + 1 || warp == W_ZERO_B || warp == W_ZERO_B + 1) {
-        // ------------------------------------------------------------------ zeros for dropped rows
-        zero_fill_dropped_rows<false, NUM_ZERO_WARPS * 32>(a.y, a.mask, g, 1, ((warp >= W_ZERO_B ? warp - W_ZERO_B + 2 : warp - W_ZERO_A) * 32 + lane));
+        // ------------------------------------------------------------------ zeros for dropped rows (a compact output has none)
+        if (!a.out_compact) zero_fill_dropped_rows<false, NUM_ZERO_WARPS * 32>(a.y, a.mask, g, 1, ((warp >= W_ZERO_B ? warp - W_ZERO_B + 2 : warp - W_ZERO_A) * 32 + lane));
     } else {
         // ------------------------------------------------------------------ A operand: patch -> tensor memory
         // Warp (quarter q, group grp) owns tile rows 32 q .. 32 q + 31 (tensor-memory lanes a warp can
@@ -610,8 +611,8 @@ void plan_patch_cost(const ConvGeom& g, int num_sms, long long n_mtiles, PatchPl
 cudaError_t launch_patch(const ConvGeom& g, const PatchPlan& plan, const CUtensorMap& tmap_w, const CUtensorMap& tmap_x4,
                          const float* bias, void* y, const uint8_t* mask, const int32_t* kept, const int32_t* count,
                          int relu, int* dev_status, int num_sms, int fuse_compact, long long host_kept,
-                         const void* residual, const void* tiles, int n_mtiles, long long kept_rows, int wait_limit_kcycles,
-                         cudaStream_t st)
+                         const void* residual, const void* tiles, int n_mtiles, long long kept_rows, int out_compact,
+                         int wait_limit_kcycles, cudaStream_t st)
 {
     PatchArgs a;
     a.fdcnt_host = make_fastdiv((uint32_t)(host_kept > 0 && host_kept < (1ll << 31) ? host_kept : 1));
@@ -627,6 +628,7 @@ cudaError_t launch_patch(const ConvGeom& g, const PatchPlan& plan, const CUtenso
     a.count = count;
     a.dev_status = dev_status;
     a.relu = relu == 1 ? 1 : 0;
+    a.out_compact = out_compact;
     a.st32 = (g.C_out % 16 == 0 && (reinterpret_cast<uintptr_t>(y) & 31) == 0) ? 1 : 0;
     a.BN = plan.BN;
     a.n_tiles = plan.n_tiles;

@@ -178,3 +178,29 @@ def test_device_masks_take_the_row_gather():
     ref = oracle.masked_conv(x, w, b, mask, 1, 1, True).reshape(spec.M, spec.C_out)
     got = out.float().cpu().numpy().astype(np.float64).reshape(spec.M, spec.C_out)
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= REL_FROB_TOL
+
+
+def test_compact_output():
+    """With ASX_OUT_COMPACT the kept rows go to y[n*P' + j] in kept order and nothing else is written."""
+    spec = spec_of("p_compact", 64, 48, 3, 3, 1, 20, 23, 3, 40, 2, seed=96)
+    x, w, b, mask = make_problem(spec)
+    kept = int(mask.sum())
+    layer = asx.MaskedConvLayer(64, 48, 3, 3, 1, 1)
+    layer.set_mask(mask)
+    y = torch.full((spec.Nb * kept + 4, spec.C_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+    st = int(torch.cuda.current_stream().cuda_stream)
+    xd, wd, bd = to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda()
+    rc = layer.run_raw(xd.data_ptr(), spec.Nb, spec.H, spec.W, wd.data_ptr(), bd.data_ptr(), y.data_ptr(),
+                       asx.ACT_RELU | asx.OUT_COMPACT | asx.IMPL_WINDOW_PATCH, st)
+    assert rc == 0
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0 and layer.last_run_form() == asx.FORM_WINDOW_PATCH
+    layer.close()
+    got = y.float().cpu().numpy().astype(np.float64)
+    assert np.isnan(got[spec.Nb * kept:]).all(), "rows behind the compact output were written"
+    rows = (np.arange(spec.Nb)[:, None] * spec.P + np.flatnonzero(mask)[None, :]).reshape(-1)
+    ref = oracle.masked_conv(x, w, b, mask, 1, 1, True).reshape(spec.M, spec.C_out)[rows]
+    got = got[:spec.Nb * kept]
+    assert not np.isnan(got).any()
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= REL_FROB_TOL
+    assert np.abs(got - ref).max() <= max_abs_tol(spec.K, oracle.bf16_round(x), oracle.bf16_round(w))
