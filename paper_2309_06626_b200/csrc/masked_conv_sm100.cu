@@ -596,24 +596,45 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                         ky = tap / g.kw;
                         kx = tap - ky * g.kw;
                     }
+                    // Compact input: the rank of every tap's input position comes from a table in global
+                    // memory.  Looked up right in front of the row gather that needs it, the load's latency
+                    // (an L2 round trip per k-block: the table competes with everything else for the little L1
+                    // the stages leave) sat in the issuing lane's serial loop and cost the layer a third of its
+                    // time; so the ranks of this lane's NEXT k-block are requested right after a gather is
+                    // issued and arrive while the lane waits for the stage after that.
+                    int rn[4] = {-1, -1, -1, -1};
+                    auto request_ranks = [&](int kbn) {
+                        const int tapn = (int)fd_div((uint32_t)(kbn * BKE), a.fdCin);
+                        const int kyn = (int)fd_div((uint32_t)tapn, a.fdkw), kxn = tapn - kyn * g.kw;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int iy = (yx[i] >> 16) + kyn, ix = (int)(short)(yx[i] & 0xffff) + kxn;
+                            const bool in = (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
+                            rn[i] = in ? __ldg(a.in_rank + iy * g.W + ix) : -1;
+                        }
+                    };
+                    if (IN_COMPACT) {
+                        const int kb0 = item.kb_lo + (((it & 1) == grp) ? 0 : 1);       // this lane's first k-block of the tile
+                        if (kb0 < item.kb_hi) request_ranks(kb0);
+                    }
                     for (int kb = item.kb_lo; kb < item.kb_hi; ++kb, ++it) {
                         if ((it & 1) == grp) {
                             const int koff = ky * g.W + kx;
                             int idx[4];
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
-                                const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
-                                const bool in = (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
                                 if (!IN_COMPACT) {
+                                    const int iy = (yx[i] >> 16) + ky, ix = (int)(short)(yx[i] & 0xffff) + kx;
+                                    const bool in = (unsigned)iy < (unsigned)g.H && (unsigned)ix < (unsigned)g.W;
                                     idx[i] = in ? pix[i] + koff : oob;
                                 } else {               // compact input: a dropped position reads zeros like padding
-                                    const int rnk = in ? __ldg(a.in_rank + iy * g.W + ix) : -1;
-                                    idx[i] = rnk >= 0 ? pix[i] + rnk : oob;
+                                    idx[i] = rn[i] >= 0 ? pix[i] + rn[i] : oob;
                                 }
                             }
                             if (!wait_bar<20>(ptx::smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, a.dev_status)) { ok = false; break; }
                             ptx::tma_gather4_2d(smem_base + s * stage_bytes + (uint32_t)(16 * pwg + 4 * lane) * 128u, &tmap_x,
                                                 ptx::smem_u32(&sh->full[s]), ci, idx[0], idx[1], idx[2], idx[3]);
+                            if (IN_COMPACT && kb + 2 < item.kb_hi) request_ranks(kb + 2);
                         }
                         ci += BKE;                         // next 128 bytes of channels, or the next tap
                         if (ci >= g.C_in) {
