@@ -41,7 +41,7 @@ L2_BYTES = 126 * 1024 * 1024
 # cold-cache and most of a launch's output is still in L2 when its counters stop).  The figure belongs to
 # the kernel sources whose digest is recorded with it; with any other sources the bench reports null.
 NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 15.18e6,
-               "csrc_sha256": "b6fbd25dddef01f1327a1001a6399723ef4734363fa01a6ffbdf82fcd5b9e3e0"}
+               "csrc_sha256": "4d9c3dd3f9dc81c6c2286f420d01471a18212b268aaf4288aac7b2b60fbd1471"}
 
 
 def csrc_digest() -> str:
@@ -435,6 +435,25 @@ def run_ours(args):
     if graph is not None:
         _, ms_median, ms_min = time_replays(graph, min(K, 200))
 
+    # ---- per-layer time in the step's own regime: the replay time of the captured prefix [0..i] minus that
+    # of [0..i-1] (in-line order, no graph branch), i.e. what layer i adds to a graph-replayed step with
+    # its set-up overlapping the previous kernel's tail as in the timed region
+    in_step_ms = None
+    if graph is not None and not args.no_marginal:
+        in_step_ms, prev = [], 0.0
+        for i in range(1, len(layers) + 1):
+            pg = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(pg):
+                cst = int(torch.cuda.current_stream().cuda_stream)
+                for L in layers[:i]:
+                    rc = L.layer.run_raw(*L.ptrs, RELU | RECOMPACT_FLAG, cst)
+                    if rc:
+                        raise RuntimeError(f"asx call failed with status {rc} during capture")
+            t = time_replays(pg, 50)[0]
+            in_step_ms.append(t - prev)
+            prev = t
+            del pg
+
     # ---- a second view: every launch of the fused kernel alone between an event pair (a spin kernel is
     # queued first so that the host runs ahead).  These per-launch times are SERIALISED: the event pair
     # keeps a launch from overlapping its neighbours, which the graph replay above allows (programmatic
@@ -730,6 +749,9 @@ def run_ours(args):
             "kernel_ms_per_step": ms_step,
             "kernel_ms_note": "the graph-replayed step: the fused kernel's launches (plus the stem's two staging kernels), "
                               "overlapping by programmatic dependent launch as in the timed region",
+            "in_step_ms_sum": None if in_step_ms is None else sum(in_step_ms),
+            "in_step_note": "per_layer.ms_in_step: replay time of the captured prefix of layers [0..i] minus that of [0..i-1]; "
+                            "sums to the step in in-line order",
             "serialised_kernel_ms_per_step": serial_ms,
             "serialised_note": "sum of per-launch times taken with an event pair around every launch (no overlap between "
                                "launches, launch gaps included): ranks the layers, exceeds the step time by construction",
@@ -764,6 +786,7 @@ def run_ours(args):
         "chain": chain,
         "sweep": sweep,
         "per_layer": [{"name": L.spec.name, "M": L.spec.M, "K": L.spec.K, "N": L.spec.N, "kept_rows": L.kept_rows,
+                       "ms_in_step": None if in_step_ms is None else in_step_ms[i],
                        "ms_serialised": per_layer_ms[i], "tflops": L.flops / (per_layer_ms[i] * 1e-3) / 1e12,
                        "gbs": L.bytes / (per_layer_ms[i] * 1e-3) / 1e9, "roof_ms": roofs[i],
                        "form": {0: "none", 1: "naive", 2: "row gather (copies)", 3: "row gather (TMA)", 4: "window patch"}[forms[i]]}
@@ -796,6 +819,7 @@ def main():
                     help="with N > 1 ranks: every rank runs the whole batch (weak, the default) or its share of the images (strong)")
     ap.add_argument("--no-fork-proj", action="store_true",
                     help="keep the 1x1 projections of down-sampling blocks in line instead of on a graph branch")
+    ap.add_argument("--no-marginal", action="store_true", help="skip the per-layer in-step times (one graph capture per layer)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":
