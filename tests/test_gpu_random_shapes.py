@@ -67,8 +67,6 @@ def test_random_geometry_window_patch(i):
     """The same kind of sweep with the window-patch form forced (300 such cases, each run three times with
     bit-identical results, were run once; this is their first 40)."""
     spec = _random_patch_spec(i)
-    rng = np.random.default_rng(555_000 + i)
-    rng.random(16)
     per_row = bool(np.random.default_rng(11 * i + 3).random() < 0.3)
     x, w, b, mask = make_problem(spec, per_row=per_row)
     flags = asx.ACT_RELU | asx.IMPL_WINDOW_PATCH | (asx.RECOMPACT if i % 2 else 0)
