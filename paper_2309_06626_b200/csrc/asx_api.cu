@@ -151,10 +151,11 @@ void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]
 }
 
 // Window-patch form: cut the kept lowered rows (ascending in image and output row) into tiles of at
-// most 128 consecutive rows whose windows span at most `cap` zero-padded input rows.  Pure index
+// most `max_rows` (<= 128) consecutive rows whose windows span at most `cap` zero-padded input rows.  Pure index
 // bookkeeping on the mask the host holds; four ints per tile (first kept lowered row, rows, first
 // padded input row of the patch, patch rows); returns the kept lowered rows, or -1 without memory.
-int64_t cut_row_tiles(const std::vector<uint8_t>& mask, int Nb, int P, int Wo, int Hp, int kh, int cap, std::vector<int32_t>* tiles)
+int64_t cut_row_tiles(const std::vector<uint8_t>& mask, int Nb, int P, int Wo, int Hp, int kh, int cap, int max_rows,
+                      std::vector<int32_t>* tiles)
 {
     std::vector<int32_t> kept;
     tiles->clear();
@@ -172,7 +173,7 @@ int64_t cut_row_tiles(const std::vector<uint8_t>& mask, int Nb, int P, int Wo, i
         for (int64_t r0 = 0; r0 < Mk;) {
             const int64_t first = padded_row(r0);
             int64_t n = 1;
-            while (n < 128 && r0 + n < Mk && padded_row(r0 + n) - first + kh <= cap) ++n;
+            while (n < max_rows && r0 + n < Mk && padded_row(r0 + n) - first + kh <= cap) ++n;
             tiles->push_back((int32_t)r0);
             tiles->push_back((int32_t)n);
             tiles->push_back((int32_t)first);                                     // first padded input row of the patch
@@ -628,7 +629,25 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     if (!f32 && !in_compact && !(flags & ASX_IMPL_ROW_GATHER) && !L->host_mask.empty() &&
         (reinterpret_cast<uintptr_t>(y) & 15) == 0 && plan_patch(g, fuse_compact ? (int)L->rows : 0, &pplan)) {
         if (L->tiles_epoch != L->mask_epoch || L->tiles_Nb != Nb || L->tiles_H != H || L->tiles_W != W || L->tiles_cap != pplan.cap_rows) {
-            L->tiles_rows = cut_row_tiles(L->host_mask, Nb, g.P, g.Wo, pplan.Hp, g.kh, pplan.cap_rows, &L->host_tiles);
+            L->tiles_rows = cut_row_tiles(L->host_mask, Nb, g.P, g.Wo, pplan.Hp, g.kh, pplan.cap_rows, 128, &L->host_tiles);
+            // Level the waves: with T tiles of 128 rows on S blocks the last of ceil(T / S) waves is partly
+            // empty; tiles of fewer rows that fill every wave cost less (a tile's patch reads and epilogue
+            // shrink with its rows, only the filter slabs do not), as long as the wave count stays.
+            if (L->tiles_rows > 0) {
+                const long long t128 = (long long)(L->host_tiles.size() / 4);
+                const long long per_wave = std::max<long long>(1, L->num_sms / pplan.n_tiles);      // row tiles one wave takes
+                const long long waves = (t128 + per_wave - 1) / per_wave;
+                const long long target = waves * per_wave;
+                if (target > t128) {
+                    int rows_per_tile = (int)((L->tiles_rows + target - 1) / target);
+                    rows_per_tile = std::min(128, (rows_per_tile + 7) / 8 * 8);
+                    std::vector<int32_t> level;
+                    if (rows_per_tile >= 32 && rows_per_tile < 128 &&
+                        cut_row_tiles(L->host_mask, Nb, g.P, g.Wo, pplan.Hp, g.kh, pplan.cap_rows, rows_per_tile, &level) == L->tiles_rows &&
+                        (long long)(level.size() / 4) <= target)
+                        L->host_tiles.swap(level);
+                }
+            }
             L->tiles_epoch = L->mask_epoch; L->tiles_Nb = Nb; L->tiles_H = H; L->tiles_W = W; L->tiles_cap = pplan.cap_rows;
             const size_t need = L->host_tiles.size() * sizeof(int32_t);
             if (L->tiles_rows > 0 && need > 0) {
