@@ -598,10 +598,9 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
                     }
                     // Compact input: the rank of every tap's input position comes from a table in global
                     // memory.  Looked up right in front of the row gather that needs it, the load's latency
-                    // (an L2 round trip per k-block: the table competes with everything else for the little L1
-                    // the stages leave) sat in the issuing lane's serial loop and cost the layer a third of its
-                    // time; so the ranks of this lane's NEXT k-block are requested right after a gather is
-                    // issued and arrive while the lane waits for the stage after that.
+                    // (the table competes with everything else for the little L1 the stages leave) sat in the
+                    // issuing lane's serial loop; so the ranks of this lane's NEXT k-block are requested right
+                    // after a gather is issued and arrive while the lane waits for the stage after that.
                     int rn[4] = {-1, -1, -1, -1};
                     auto request_ranks = [&](int kbn) {
                         const int tapn = (int)fd_div((uint32_t)(kbn * BKE), a.fdCin);
