@@ -61,6 +61,7 @@ struct asx_layer {
     CUtensorMap tmap_x4;               // x as a 4-D tensor (C_in, W, H, Nb) with one padded row of 64 channels per box
     const void* tmapx4_ptr = nullptr;
     int tmapx4_Nb = 0, tmapx4_H = 0, tmapx4_W = 0, tmapx4_Wp = 0;
+    int tmapx4_px32 = 0;
     int wait_limit_kcycles = 0;
     int last_form = ASX_FORM_NONE;     // producer form of the last asx_run        // bound of the in-kernel waits in units of 1024 cycles (0: the default, about 2 s)
 };
@@ -502,7 +503,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         const int kh2 = (L->kh + bshift + 1) / 2;
         const int h0 = (L->pad + bshift) / 2;                              // border on the top and left, in blocks
         const int Hs = (h0 + H / 2 > g.Ho + kh2 - 1) ? h0 + H / 2 : g.Ho + kh2 - 1;
-        const int Ws = (h0 + W / 2 > g.Wo + 3) ? h0 + W / 2 : g.Wo + 3;
+        const int Ws = (((h0 + W / 2 > g.Wo + 3) ? h0 + W / 2 : g.Wo + 3) + 3) / 4 * 4;     // whole 128-byte units of four blocks
         const int64_t nblocks = (int64_t)Nb * Hs * Ws;
         if (nblocks * 16 > lim) return ASX_ERR_UNSUPPORTED;
         const size_t need_x = (size_t)nblocks * 32 + 128, need_w = (size_t)L->C_out * kh2 * 64 * 2;
@@ -626,10 +627,16 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     // estimate favours it; compact inputs and fp32 storage stay with the row gather.
     PatchPlan pplan;
     bool use_patch = false;
+    // The window-patch kernel sees the input as [Nb][H][W] pixels of C_in channels.  In the 2x2-block form a
+    // "pixel" is the 128-byte run of four blocks that starts at a block, pixels are 32 bytes apart (they
+    // overlap); the patch holds every block once, Wo + 3 per row, and only the first Ho + kh - 1 block rows
+    // are ever read.
+    ConvGeom gp = g;
+    if (blocks2x2) gp.H = g.Ho + g.kh - 1;
     if (!f32 && !in_compact && !(flags & ASX_IMPL_ROW_GATHER) && !L->host_mask.empty() &&
-        (reinterpret_cast<uintptr_t>(y) & 15) == 0 && plan_patch(g, fuse_compact ? (int)L->rows : 0, &pplan)) {
+        (reinterpret_cast<uintptr_t>(y) & 15) == 0 && plan_patch(gp, fuse_compact ? (int)L->rows : 0, blocks2x2 ? 1 : 0, &pplan)) {
         if (L->tiles_epoch != L->mask_epoch || L->tiles_Nb != Nb || L->tiles_H != H || L->tiles_W != W || L->tiles_cap != pplan.cap_rows) {
-            L->tiles_rows = cut_row_tiles(L->host_mask, Nb, g.P, g.Wo, pplan.Hp, g.kh, pplan.cap_rows, 128, &L->host_tiles);
+            L->tiles_rows = cut_row_tiles(L->host_mask, Nb, gp.P, gp.Wo, pplan.Hp, gp.kh, pplan.cap_rows, 128, &L->host_tiles);
             // Level the waves: with T tiles of 128 rows on S blocks the last of ceil(T / S) waves is partly
             // empty; tiles of fewer rows that fill every wave cost less (a tile's patch reads and epilogue
             // shrink with its rows, only the filter slabs do not), as long as the wave count stays.
@@ -643,7 +650,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
                     rows_per_tile = std::min(128, (rows_per_tile + 7) / 8 * 8);
                     std::vector<int32_t> level;
                     if (rows_per_tile >= 32 && rows_per_tile < 128 &&
-                        cut_row_tiles(L->host_mask, Nb, g.P, g.Wo, pplan.Hp, g.kh, pplan.cap_rows, rows_per_tile, &level) == L->tiles_rows &&
+                        cut_row_tiles(L->host_mask, Nb, gp.P, gp.Wo, pplan.Hp, gp.kh, pplan.cap_rows, rows_per_tile, &level) == L->tiles_rows &&
                         (long long)(level.size() / 4) <= target)
                         L->host_tiles.swap(level);
                 }
@@ -664,7 +671,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
             }
         }
         if (L->tiles_rows > 0 && L->tiles_rows == est_rows) {
-            plan_patch_cost(g, L->num_sms, (long long)(L->host_tiles.size() / 4), &pplan);
+            plan_patch_cost(gp, L->num_sms, (long long)(L->host_tiles.size() / 4), &pplan);
             use_patch = pplan.est_cost_us <= plan.est_cost_us || (flags & ASX_IMPL_WINDOW_PATCH);
         }
     }
@@ -703,21 +710,26 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
         L->tmap_ptr = wsrc; L->tmap_BN = BNsel; L->tmap_Kw = Kw; L->tmap_es = ES;
     }
     if (use_patch) {
-        if (L->tmapx4_ptr != xsrc || L->tmapx4_Nb != Nb || L->tmapx4_H != g.H || L->tmapx4_W != g.W || L->tmapx4_Wp != pplan.Wp) {
+        if (L->tmapx4_ptr != xsrc || L->tmapx4_Nb != Nb || L->tmapx4_H != g.H || L->tmapx4_W != g.W || L->tmapx4_Wp != pplan.Wp ||
+            L->tmapx4_px32 != pplan.px32) {
             EncodeTiledFn enc = encode_tiled_fn();
             if (enc == nullptr) return ASX_ERR_CUDA;
-            const cuuint64_t dims[4] = {(cuuint64_t)g.C_in, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)Nb};
-            const cuuint64_t strides[3] = {(cuuint64_t)g.C_in * 2, (cuuint64_t)g.W * g.C_in * 2, (cuuint64_t)g.H * g.W * g.C_in * 2};
+            // g.H x g.W pixels of g.C_in channels; in the 2x2-block form block rows of g.W / 4 units of four blocks
+            // (64 values), which the box takes whole
+            const cuuint64_t wu = pplan.px32 ? (cuuint64_t)g.W / 4 : (cuuint64_t)g.W;
+            const cuuint64_t dims[4] = {(cuuint64_t)g.C_in, wu, (cuuint64_t)g.H, (cuuint64_t)Nb};
+            const cuuint64_t strides[3] = {(cuuint64_t)g.C_in * 2, wu * g.C_in * 2, (cuuint64_t)g.H * wu * g.C_in * 2};
             const cuuint32_t box[4] = {64u, (cuuint32_t)pplan.Wp, 1u, 1u};
             const cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
             const CUresult r = enc(&L->tmap_x4, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(xsrc), dims, strides, box, estr,
-                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) return ASX_ERR_CUDA;
             L->tmapx4_ptr = xsrc; L->tmapx4_Nb = Nb; L->tmapx4_H = g.H; L->tmapx4_W = g.W; L->tmapx4_Wp = pplan.Wp;
+            L->tmapx4_px32 = pplan.px32;
         }
         L->last_form = ASX_FORM_WINDOW_PATCH;
-        return from_cuda(launch_patch(g, pplan, L->tmap, L->tmap_x4, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status, L->num_sms,
+        return from_cuda(launch_patch(gp, pplan, L->tmap, L->tmap_x4, bias, y, L->d_mask, L->d_kept, d_count, relu, d_status, L->num_sms,
                                       fuse_compact ? 1 : 0, L->host_kept, L->residual, L->d_tiles, (int)(L->host_tiles.size() / 4), L->tiles_rows,
                                       out_compact ? 1 : 0, L->wait_limit_kcycles, st));
     }

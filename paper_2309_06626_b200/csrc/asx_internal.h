@@ -86,14 +86,19 @@ struct PatchPlan {
     int G;                 // filter taps per pipeline stage
     int cap_rows;          // padded input rows one patch buffer holds: every tile's windows must span at most this many
     int Hp, Wp, Wp8;       // padded input height and width, Wp rounded up to a multiple of 8
+    int p_bufs_log2;       // 1 or 2: two or four patch buffers of cap_rows rows
+    int epi8;              // eight epilogue warps and twelve fill warps instead of four and sixteen
+    int px32;              // pixels are overlapping runs of four 32-byte blocks (the 2x2-block form of a first layer)
     int smem_bytes;
     double est_cost_us;    // the planner's estimate of the launch's duration
 };
 // false: this geometry does not take the window-patch form
-bool plan_patch(const ConvGeom& g, int fused_list_rows, PatchPlan* plan);
+// px32: g describes the 2x2-block form (64 channels = four 32-byte blocks, kw = 1, no padding, pixels 32 bytes apart)
+bool plan_patch(const ConvGeom& g, int fused_list_rows, int px32, PatchPlan* plan);
 // fills plan->est_cost_us for a mask that the host cut into n_mtiles row tiles
 void plan_patch_cost(const ConvGeom& g, int num_sms, long long n_mtiles, PatchPlan* plan);
-// tmap_x4: x as a 4-D tensor (C_in, W, H, Nb) with box (64, Wp, 1, 1), 128-byte swizzle, zero fill
+// tmap_x4: x as a 4-D tensor (C_in, W, H, Nb) with box (64, Wp, 1, 1), 128-byte swizzle, zero fill; for a px32 plan
+// W counts units of four blocks (64 values)
 cudaError_t launch_patch(const ConvGeom& g, const PatchPlan& plan, const CUtensorMap& tmap_w, const CUtensorMap& tmap_x4,
                          const float* bias, void* y, const uint8_t* mask, const int32_t* kept, const int32_t* count,
                          int relu, int* dev_status, int num_sms, int fuse_compact, long long host_kept,

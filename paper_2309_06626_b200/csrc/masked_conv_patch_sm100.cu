@@ -45,6 +45,7 @@ constexpr int INFO_RING = 8;            // tiles whose row coordinates are kept 
 constexpr int MAX_B_STAGES = 8;
 constexpr int MAX_A_STAGES = 12;
 constexpr int TAP_COLS = 32;            // 64 bf16 per row = 32 columns of tensor memory per filter tap
+constexpr int MAX_P_BUFS = 4;           // patch buffers: two, or four where four still hold a tile's rows each
 constexpr int FULL_RING = 24;           // 'stage full' barriers: a multiple of every A and filter ring depth in use (2, 3, 4)
 // Warp roles.  The two loader warps come last: they take no part in the mask compaction and the row
 // decoding (threads 0 .. WORK_THREADS-1 do, meeting on hardware barrier 2) but start fetching filter
@@ -72,7 +73,14 @@ struct PatchArgs {
     int st32;           // 32-byte epilogue stores: C_out % 16 == 0, BN % 16 == 0 and y 32-byte aligned
     int BN, n_tiles, b_stages, a_stages;
     int cap_rows;       // padded input rows one patch buffer holds
+    int p_bufs_log2;    // 1 or 2: two or four patch buffers
+    int epi8;           // few k-blocks per tile: the last four fill warps are epilogue warps too (each warp of a lane
+                        // quarter's pair takes every other 32-column chunk), three fill groups remain
     int Hp, Wp, Wp8;    // padded input height and width; Wp rounded up to a multiple of 8 (row pitch in pixels)
+    int px32;           // 2x2-block form of a network's first layer: a "pixel" is a 32-byte block, a window row is the
+                        // 128 bytes of four consecutive blocks (kw = 1), so neighbouring pixels overlap; the patch holds
+                        // each block once instead of 128 bytes per pixel: Wp counts the 128-byte units (four blocks) a
+                        // row's box has, Wp8 the row pitch in blocks (a multiple of 32: rows start 1024-byte aligned)
     int slices;         // C_in / 64
     int G;              // filter taps per pipeline stage (a chunk); chunks = ceil(kh*kw / G) per slice
     int fuse_compact;   // rebuild the kept-row list from the mask inside this kernel (small masks)
@@ -97,8 +105,8 @@ struct alignas(16) PShared {          // lives after the patch buffers and the f
     unsigned long long full[FULL_RING];
     unsigned long long b_empty[MAX_B_STAGES];
     unsigned long long a_empty[MAX_A_STAGES];
-    unsigned long long p_full[2];
-    unsigned long long p_empty[2];
+    unsigned long long p_full[MAX_P_BUFS];
+    unsigned long long p_empty[MAX_P_BUFS];
     unsigned long long acc_full[2];
     unsigned long long acc_empty[2];
     unsigned int tmem_base;
@@ -172,13 +180,15 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
     const int chunks = (taps + G - 1) / G;                            // pipeline stages per slice
     const int NST = chunks * a.slices;                                // pipeline stages per work item
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t row_bytes = (uint32_t)a.Wp8 * 128u;                // one padded input row of one slice
-    const uint32_t patch_bytes = (uint32_t)a.cap_rows * row_bytes;    // a multiple of 1024
-    const uint32_t b_base = smem_base + 2u * patch_bytes;
+    const uint32_t px_bytes = a.px32 ? 32u : 128u;
+    const uint32_t row_bytes = (uint32_t)a.Wp8 * px_bytes;            // one padded input row of one slice
+    const uint32_t patch_bytes = ((uint32_t)a.cap_rows * row_bytes + 1023u) & ~1023u;
+    const uint32_t PB = 1u << a.p_bufs_log2;                         // patch buffers (2 or 4)
+    const uint32_t b_base = smem_base + PB * patch_bytes;
     const uint32_t b_tap_bytes = (uint32_t)BN * 128u;                 // the filter slab of one tap of one slice
     const uint32_t b_stage_bytes = (uint32_t)G * b_tap_bytes;
     const uint32_t a_stage_cols = (uint32_t)(G * TAP_COLS);
-    PShared* sh = reinterpret_cast<PShared*>(smem_raw + (smem_base - ptx::smem_u32(smem_raw)) + 2u * patch_bytes + (uint32_t)BS * b_stage_bytes);
+    PShared* sh = reinterpret_cast<PShared*>(smem_raw + (smem_base - ptx::smem_u32(smem_raw)) + PB * patch_bytes + (uint32_t)BS * b_stage_bytes);
     volatile WaitCtl* ctl = &sh->ctl;
 
     uint4 early_mask = make_uint4(0, 0, 0, 0);
@@ -187,7 +197,7 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
 
     // barrier initialisation, one barrier per thread (a single thread took about 1500 clocks over them)
     {
-        constexpr int NB = FULL_RING + MAX_B_STAGES + MAX_A_STAGES + 2 * INFO_RING + 8;
+        constexpr int NB = FULL_RING + MAX_B_STAGES + MAX_A_STAGES + 2 * INFO_RING + 2 * MAX_P_BUFS + 4;
         if (tid < NB) {
             int i = tid;
             unsigned long long* bar;
@@ -196,11 +206,11 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
             else if ((i -= FULL_RING) < MAX_B_STAGES) { bar = &sh->b_empty[i]; count = 1; }
             else if ((i -= MAX_B_STAGES) < MAX_A_STAGES) { bar = &sh->a_empty[i]; count = 1; }
             else if ((i -= MAX_A_STAGES) < INFO_RING) { bar = &sh->info_full[i]; count = 1; }
-            else if ((i -= INFO_RING) < INFO_RING) { bar = &sh->info_empty[i]; count = NUM_FILL_WARPS; }
-            else if ((i -= INFO_RING) < 2) { bar = &sh->p_full[i]; count = 1; }
-            else if ((i -= 2) < 2) { bar = &sh->p_empty[i]; count = NUM_FILL_WARPS; }
-            else if ((i -= 2) < 2) { bar = &sh->acc_full[i]; count = 1; }
-            else { i -= 2; bar = &sh->acc_empty[i]; count = NUM_EPI_WARPS; }
+            else if ((i -= INFO_RING) < INFO_RING) { bar = &sh->info_empty[i]; count = a.epi8 ? NUM_FILL_WARPS - 4 : NUM_FILL_WARPS; }
+            else if ((i -= INFO_RING) < MAX_P_BUFS) { bar = &sh->p_full[i]; count = 1; }
+            else if ((i -= MAX_P_BUFS) < MAX_P_BUFS) { bar = &sh->p_empty[i]; count = a.epi8 ? NUM_FILL_WARPS - 4 : NUM_FILL_WARPS; }
+            else if ((i -= MAX_P_BUFS) < 2) { bar = &sh->acc_full[i]; count = 1; }
+            else { i -= 2; bar = &sh->acc_empty[i]; count = a.epi8 ? 2 * NUM_EPI_WARPS : NUM_EPI_WARPS; }
             ptx::mbar_init(ptx::smem_u32(bar), count);
             ptx::fence_mbar_init();
         }
@@ -236,6 +246,10 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
                 // Stages run slice by slice (all taps of channels 64 s .. 64 s + 63, then the next slice),
                 // so that one slice of the patch is in use at a time; in w[C_out][kh][kw][C_in] the slab
                 // of (tap, slice) starts at K index tap * C_in + 64 * slice.
+                // When the ring holds a whole work item's stages and there is one column tile, stage s always
+                // gets the same slab: it is loaded for the block's first tile only and stays (the stage's
+                // barrier still gets this thread's arrival, in step with the MMA warp's releases).
+                const bool resident = (NST == BS && a.n_tiles == 1);
                 int s = 0, fi = 0;
                 uint32_t ph = 0;
                 for (int t = blockIdx.x; t < host_tiles && ok; t += gridDim.x) {
@@ -245,10 +259,14 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
                             const int gc = taps - tap0 < G ? taps - tap0 : G;
                             if (!wait_bar<40>(ptx::smem_u32(&sh->b_empty[s]), ph ^ 1u, ctl, a.dev_status)) { ok = false; break; }
                             const uint32_t full = ptx::smem_u32(&sh->full[fi]);
-                            ptx::mbar_arrive_expect_tx(full, (uint32_t)gc * b_tap_bytes);
-                            for (int i = 0; i < gc; ++i)
-                                ptx::tma_load_2d(b_base + (uint32_t)s * b_stage_bytes + (uint32_t)i * b_tap_bytes, &tmap_w, full,
-                                                 (tap0 + i) * g.C_in + sl * 64, n_tile * BN);
+                            if (resident && t != (int)blockIdx.x) {
+                                ptx::mbar_arrive(full);
+                            } else {
+                                ptx::mbar_arrive_expect_tx(full, (uint32_t)gc * b_tap_bytes);
+                                for (int i = 0; i < gc; ++i)
+                                    ptx::tma_load_2d(b_base + (uint32_t)s * b_stage_bytes + (uint32_t)i * b_tap_bytes, &tmap_w, full,
+                                                     (tap0 + i) * g.C_in + sl * 64, n_tile * BN);
+                            }
                             if (++s == BS) { s = 0; ph ^= 1u; }
                             if (++fi == FULL_RING) fi = 0;
                         }
@@ -268,8 +286,8 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
                     }
                     const int n_lo = (int)fd_div((uint32_t)tl.z, a.fdHp);
                     for (int sl = 0; sl < a.slices; ++sl, ++use) {
-                        const uint32_t b = use & 1u;
-                        if (!wait_bar<40>(ptx::smem_u32(&sh->p_empty[b]), ((use >> 1) & 1u) ^ 1u, ctl, a.dev_status)) { ok = false; break; }
+                        const uint32_t b = use & (PB - 1u);
+                        if (!wait_bar<40>(ptx::smem_u32(&sh->p_empty[b]), ((use >> a.p_bufs_log2) & 1u) ^ 1u, ctl, a.dev_status)) { ok = false; break; }
                         const uint32_t full = ptx::smem_u32(&sh->p_full[b]);
                         ptx::mbar_arrive_expect_tx(full, (uint32_t)nrows * (uint32_t)a.Wp * 128u);
                         int n = n_lo, yy = tl.z - n_lo * a.Hp;             // padded row yy of image n
@@ -386,9 +404,12 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
             if (ok && ptx::elect_one()) ptx::umma_commit(ptx::smem_u32(&sh->acc_full[buf]));
             __syncwarp();
         }
-    } else if (warp >= W_EPI0 && warp < W_EPI0 + NUM_EPI_WARPS) {
+    } else if ((warp >= W_EPI0 && warp < W_EPI0 + NUM_EPI_WARPS) || (a.epi8 && warp >= W_FILL0 + NUM_FILL_WARPS - 4 && warp < W_FILL0 + NUM_FILL_WARPS)) {
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3;                       // TMEM lanes 32q .. 32q+31 belong to this warp
+        const int half = warp >= W_FILL0 ? 1 : 0;     // with eight epilogue warps: which of the pair this one is
+        const int epi_threads = a.epi8 ? 2 * NUM_EPI_WARPS * 32 : NUM_EPI_WARPS * 32;
+        const int c_step = a.epi8 ? 64 : 32;
         unsigned short* y2 = reinterpret_cast<unsigned short*>(a.y);
         int ti = 0;
         bool ok = true;
@@ -403,15 +424,15 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
             const long long yoff = valid ? (long long)(a.out_compact ? rk : out_row_of(rk, fdcnt, g, kept_list)) * N : 0;
             {
                 float* sb = sh->bias[buf];
-                const int et = (warp - W_EPI0) * 32 + lane;
+                const int et = half * (NUM_EPI_WARPS * 32) + q * 32 + lane;
                 if (et < BN) sb[et] = (a.bias != nullptr && n0 + et < N) ? __ldg(a.bias + n0 + et) : 0.f;
-                asm volatile("bar.sync 1, %0;" ::"n"(NUM_EPI_WARPS * 32) : "memory");
+                asm volatile("bar.sync 1, %0;" ::"r"(epi_threads) : "memory");
             }
             const float* sbias = sh->bias[buf];
             if (!warp_wait_bar<100>(ptx::smem_u32(&sh->acc_full[buf]), use, ctl, a.dev_status)) { ok = false; break; }
             ptx::tc_fence_after_sync();
             const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int c0 = half * 32; c0 < BN; c0 += c_step) {
                 const int col0 = n0 + c0;
                 if (col0 >= N) break;
                 uint32_t r[32];
@@ -475,6 +496,10 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
         }
     } else if (warp == W_ZERO_A || warp == W_ZERO_A + 1 || warp == W_ZERO_B || warp == W_ZERO_B + 1) {
         // ------------------------------------------------------------------ zeros for dropped rows (a compact output has none)
+        // Each block zeroes a fixed share of the output rows, independent of the tile loop.  (Zeroing tile by
+        // tile - the dropped rows between a tile's first kept row and the next tile's, so that a stretch of the
+        // output leaves one SM at one time - was measured: the short ranges are all latency, 87 us against 71
+        // on the first layer.)
         if (!a.out_compact) zero_fill_dropped_rows<false, NUM_ZERO_WARPS * 32>(a.y, a.mask, g, 1, ((warp >= W_ZERO_B ? warp - W_ZERO_B + 2 : warp - W_ZERO_A) * 32 + lane));
     } else {
         // ------------------------------------------------------------------ A operand: patch -> tensor memory
@@ -486,10 +511,10 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
         const int q = warp & 3, grp = (warp - W_FILL0) >> 2;
         const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + a_col0;
         // every tap of a row must stay inside the buffer even if the plan were wrong
-        const int max_base = a.cap_rows * a.Wp8 - ((g.kh - 1) * a.Wp8 + g.kw);
+        const int max_base = a.cap_rows * a.Wp8 - ((g.kh - 1) * a.Wp8 + (a.px32 ? 4 : g.kw));
         uint32_t it = 0, use = 0, aph = 0;          // stage counter of the launch, its A stage and phase
         int as = 0, fi = 0, j = 0, gsel = 0;
-        const int NG = AS < 4 ? AS : 4;
+        const int NG = a.epi8 ? 3 : (AS < 4 ? AS : 4);
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++j) {
             const int r = j & (INFO_RING - 1);
@@ -500,8 +525,8 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
             int base = px >= 0 ? px : 0;                                           // rows past the end read pixel 0; their results are never stored
             base = base < 0 ? 0 : (base > max_base ? max_base : base);
             for (int sl = 0; sl < a.slices && ok; ++sl, ++use) {
-                const uint32_t b = use & 1u;
-                if (!warp_wait_bar<20>(ptx::smem_u32(&sh->p_full[b]), (use >> 1) & 1u, ctl, a.dev_status)) { ok = false; break; }
+                const uint32_t b = use & (PB - 1u);
+                if (!warp_wait_bar<20>(ptx::smem_u32(&sh->p_full[b]), (use >> a.p_bufs_log2) & 1u, ctl, a.dev_status)) { ok = false; break; }
                 const uint32_t pb = smem_base + b * patch_bytes;
                 int ky = 0, kx = 0;
                 for (int tap0 = 0; tap0 < taps; tap0 += G, ++it) {
@@ -514,12 +539,24 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
 #pragma unroll 1
                         for (int i = 0; i < gc; ++i) {
                             const int pix = base + kyi * a.Wp8 + kxi;
-                            const uint32_t src = pb + (uint32_t)pix * 128u;
-                            const uint32_t sw = (uint32_t)(pix & 7);
                             uint32_t v[32];
+                            if (a.px32) {
+                                // blocks pix .. pix + 3, 16 bytes at a time, through the 128-byte swizzle of the rows
+                                // (1024-byte aligned): it is also what keeps eight neighbouring rows' reads, 32 bytes
+                                // apart, on different banks
+                                const uint32_t off = (uint32_t)pix * 32u;
 #pragma unroll
-                            for (int c = 0; c < 8; ++c)
-                                ptx::ld_shared_v4(src + (((uint32_t)c ^ sw) << 4), v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+                                for (int c = 0; c < 8; ++c) {
+                                    const uint32_t o = off + (uint32_t)c * 16u;
+                                    ptx::ld_shared_v4(pb + (o ^ ((o >> 3) & 0x70u)), v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+                                }
+                            } else {
+                                const uint32_t src = pb + (uint32_t)pix * 128u;
+                                const uint32_t sw = (uint32_t)(pix & 7);
+#pragma unroll
+                                for (int c = 0; c < 8; ++c)
+                                    ptx::ld_shared_v4(src + (((uint32_t)c ^ sw) << 4), v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+                            }
                             ptx::tmem_st_32(tdst + (uint32_t)(i * TAP_COLS), v);
                             if (++kxi == g.kw) { kxi = 0; ++kyi; }
                         }
@@ -555,13 +592,17 @@ int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
 }  // namespace
 
-bool plan_patch(const ConvGeom& g, int fused_list_rows, PatchPlan* plan)
+bool plan_patch(const ConvGeom& g, int fused_list_rows, int px32, PatchPlan* plan)
 {
     if (g.stride != 1 || g.stride_w != 1 || g.C_in % 64 != 0 || g.kh * g.kw < 2 || g.C_out % 8 != 0) return false;
-    const int Wp = g.W + 2 * g.pad_w, Hp = g.H + 2 * g.pad;
+    if (px32 && (g.C_in != 64 || g.kw != 1 || g.pad != 0 || g.pad_w != 0)) return false;
+    // px32: a patch row holds the Wo + 3 blocks that the row's windows touch, loaded as whole 128-byte units of
+    // four blocks (the staged rows are a multiple of four blocks long)
+    const int Wp = px32 ? (g.Wo + 3 + 3) / 4 : g.W + 2 * g.pad_w, Hp = g.H + 2 * g.pad;
+    if (px32 && (g.W % 4 != 0 || Wp * 4 > g.W)) return false;
     if (Wp > 256 || g.kh > Hp || g.kw > Wp) return false;
     // Hp and Wp as the kernel uses them need the output to be the full stride-1 range
-    if (g.Ho != Hp - g.kh + 1 || g.Wo != Wp - g.kw + 1) return false;
+    if (g.Ho != Hp - g.kh + 1 || (!px32 && g.Wo != Wp - g.kw + 1)) return false;
     const int N = g.C_out;
     const int n_tiles = (N + 127) / 128;
     const int BN = round_up((N + n_tiles - 1) / n_tiles, 16);
@@ -571,14 +612,35 @@ bool plan_patch(const ConvGeom& g, int fused_list_rows, PatchPlan* plan)
     int G = BN <= 32 ? 4 : BN <= 64 ? 3 : 2;
     if (g.kh * g.kw < G) G = g.kh * g.kw;
     while (G > 1 && (512 - 2 * BN) / (G * TAP_COLS) < 2) --G;
+    if (px32 && G > 2 && (g.kh * g.kw) % G != 0 && (g.kh * g.kw) % (G - 1) == 0) --G;      // four taps: two even stages
+    const int Wp8 = px32 ? round_up(Wp * 4, 32) : round_up(Wp, 8);      // row pitch in pixels: rows start 1024-byte aligned
+    const int px_bytes = px32 ? 32 : 128;
+    const int list_bytes = (fused_list_rows * 2 + 15) / 16 * 16;
+    // Wide rows (the 112-pixel rows of a network's first layer are 14 KB each) leave few patch rows beside
+    // three filter stages; a tile should span at least three output rows, or most of its 128 rows stay
+    // empty.  Then the filter ring shrinks first to stages of two taps, then to two stages.
+    int b_stages = 3, cap_rows = 0, half = 0;
+    for (int attempt = 0; attempt < 3; ++attempt) {
+        if (attempt == 1) { if (G <= 2) continue; G = 2; }
+        if (attempt == 2) b_stages = 2;
+        if (px32 && (g.kh * g.kw) % G == 0 && (g.kh * g.kw) / G <= 3) b_stages = (g.kh * g.kw) / G;     // the whole filter stays in the ring
+        const int budget = 227 * 1024 - 1024 - (int)sizeof(PShared) - list_bytes - b_stages * G * BN * 128;
+        half = budget < 0 ? 0 : budget / 2 / 1024 * 1024;                // a buffer is a multiple of 1024 bytes
+        cap_rows = half / (Wp8 * px_bytes);
+        if (cap_rows >= g.kh + 2) break;
+    }
+    // The rows of the 2x2-block form are short (a quarter of a 128-byte-per-pixel row), a tile's patch is a
+    // few KB and arrives after one memory latency: four buffers keep three loads in flight instead of one.
+    int p_bufs_log2 = 1;
+    if (px32 && (half / 2 / 1024 * 1024) / (Wp8 * px_bytes) >= g.kh + 4) { p_bufs_log2 = 2; cap_rows = (half / 2 / 1024 * 1024) / (Wp8 * px_bytes); }
+    if (cap_rows > 64) cap_rows = 64;
     int a_stages = (512 - 2 * BN) / (G * TAP_COLS);
     if (a_stages > 4) a_stages = 4;             // ring depths divide FULL_RING
+    // Up to four k-blocks per tile: the epilogue, not the main loop, sets the pace, so four of the sixteen fill
+    // warps join it; the twelve that remain are three groups, which take three A stages.
+    const int epi8 = (g.kh * g.kw * (g.C_in / 64) <= 4 && BN % 64 == 0 && a_stages >= 3) ? 1 : 0;
+    if (epi8) a_stages = 3;
     if (a_stages < 2) return false;
-    const int b_stages = 3;
-    const int Wp8 = round_up(Wp, 8);
-    const int list_bytes = (fused_list_rows * 2 + 15) / 16 * 16;
-    const int budget = 227 * 1024 - 1024 - (int)sizeof(PShared) - list_bytes - b_stages * G * BN * 128;
-    const int cap_rows = budget / 2 / (Wp8 * 128);
     if (cap_rows < g.kh) return false;
     plan->BN = BN;
     plan->n_tiles = (N + BN - 1) / BN;
@@ -589,7 +651,10 @@ bool plan_patch(const ConvGeom& g, int fused_list_rows, PatchPlan* plan)
     plan->Hp = Hp;
     plan->Wp = Wp;
     plan->Wp8 = Wp8;
-    plan->smem_bytes = 1024 + 2 * cap_rows * Wp8 * 128 + b_stages * G * BN * 128 + (int)sizeof(PShared) + list_bytes;
+    plan->px32 = px32;
+    plan->p_bufs_log2 = p_bufs_log2;
+    plan->epi8 = epi8;
+    plan->smem_bytes = 1024 + (1 << p_bufs_log2) * round_up(cap_rows * Wp8 * px_bytes, 1024) + b_stages * G * BN * 128 + (int)sizeof(PShared) + list_bytes;
     plan->est_cost_us = 0.0;          // set by plan_patch_cost once the tiles are cut
     return true;
 }
@@ -639,6 +704,9 @@ cudaError_t launch_patch(const ConvGeom& g, const PatchPlan& plan, const CUtenso
     a.Hp = plan.Hp;
     a.Wp = plan.Wp;
     a.Wp8 = plan.Wp8;
+    a.px32 = plan.px32;
+    a.p_bufs_log2 = plan.p_bufs_log2;
+    a.epi8 = plan.epi8;
     a.slices = g.C_in / 64;
     a.fuse_compact = fuse_compact;
     a.kept_out = const_cast<int32_t*>(kept);

@@ -204,3 +204,37 @@ def test_compact_output():
     assert not np.isnan(got).any()
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= REL_FROB_TOL
     assert np.abs(got - ref).max() <= max_abs_tol(spec.K, oracle.bf16_round(x), oracle.bf16_round(w))
+
+
+STEM_CASES = [
+    # name, C_in, C_out, k, pad, H, W, Nb, pct, block: stride-2 first layers, which reach the window-patch form
+    # through the 2x2-block staging (pixels are overlapping runs of four 32-byte blocks)
+    ("stem_7x7_c3_64", 3, 64, 7, 3, 64, 64, 2, 50, 4),
+    ("stem_7x7_c3_224", 3, 64, 7, 3, 224, 224, 1, 50, 4),         # the ResNet stem: four patch buffers, eight epilogue warps
+    ("stem_7x7_c3_n32", 3, 32, 7, 3, 32, 48, 3, 30, 1),
+    ("stem_7x7_c3_dense", 3, 64, 7, 3, 96, 160, 2, 0, 1),
+    ("stem_7x7_c1_n16", 1, 16, 7, 3, 40, 40, 2, 75, 4),
+    ("stem_7x7_c3_n128", 3, 128, 7, 3, 64, 64, 2, 50, 4),
+    ("stem_7x7_c3_pad2", 3, 64, 7, 2, 64, 64, 2, 50, 4),
+    ("stem_7x7_c4_w_odd_blocks", 4, 64, 7, 3, 36, 52, 2, 40, 2),  # staged rows padded up to whole 128-byte units
+]
+
+
+@pytest.mark.parametrize("case", STEM_CASES, ids=[c[0] for c in STEM_CASES])
+@pytest.mark.parametrize("recompact", [False, True], ids=["stored_list", "recompact"])
+def test_first_layer_in_the_window_patch_form(case, recompact):
+    name, cin, cout, k, pad, H, W, Nb, pct, blk = case
+    spec = wl.LayerSpec(name, cin, cout, k, k, 2, pad, H, W, Nb, pct, blk, "relu", wl.BASE_SEED + 7700 + len(name))
+    x, w, b, mask = make_problem(spec, per_row=False)
+    flags = asx.ACT_RELU | asx.IMPL_WINDOW_PATCH | (asx.RECOMPACT if recompact else 0)
+    check_against_oracle(spec, x, w, b, mask, flags)
+    _, bits_p, form_p = run_form(spec, x, w, b, mask, flags)
+    assert form_p == asx.FORM_WINDOW_PATCH
+    # and the row-gather form of the same staged problem gives the same bits (same products, same order of k-blocks)
+    _, bits_g, form_g = run_form(spec, x, w, b, mask, (flags & ~asx.IMPL_WINDOW_PATCH) | asx.IMPL_ROW_GATHER)
+    assert form_g != asx.FORM_WINDOW_PATCH
+    fm = (mask if mask.size == spec.M else np.tile(mask, spec.Nb)).astype(bool)
+    assert not np.any(bits_p[~fm]) and not np.any(bits_g[~fm])
+    yp = torch.from_numpy(bits_p.view(np.int16)).view(torch.bfloat16).float().numpy()
+    yg = torch.from_numpy(bits_g.view(np.int16)).view(torch.bfloat16).float().numpy()
+    assert np.max(np.abs(yp - yg)) <= 2.0 ** -6 * max(1.0, float(np.max(np.abs(yg))))
