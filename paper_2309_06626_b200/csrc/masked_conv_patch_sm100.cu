@@ -612,7 +612,11 @@ bool plan_patch(const ConvGeom& g, int fused_list_rows, int px32, PatchPlan* pla
     int G = BN <= 32 ? 4 : BN <= 64 ? 3 : 2;
     if (g.kh * g.kw < G) G = g.kh * g.kw;
     while (G > 1 && (512 - 2 * BN) / (G * TAP_COLS) < 2) --G;
-    if (px32 && G > 2 && (g.kh * g.kw) % G != 0 && (g.kh * g.kw) % (G - 1) == 0) --G;      // four taps: two even stages
+    // 2x2-block form: a tile has only kh taps (four for a 7- or 8-wide filter), so the per-stage and per-tile
+    // bookkeeping of the issuing thread and the fill warps weighs as much as the work; all taps in one stage
+    // when three A stages of that size fit beside the accumulators.
+    if (px32 && g.kh * g.kw <= 4 && (512 - 2 * BN) / (g.kh * g.kw * TAP_COLS) >= 3) G = g.kh * g.kw;
+    else if (px32 && G > 2 && (g.kh * g.kw) % G != 0 && (g.kh * g.kw) % (G - 1) == 0) --G;
     const int Wp8 = px32 ? round_up(Wp * 4, 32) : round_up(Wp, 8);      // row pitch in pixels: rows start 1024-byte aligned
     const int px_bytes = px32 ? 32 : 128;
     const int list_bytes = (fused_list_rows * 2 + 15) / 16 * 16;
