@@ -195,11 +195,12 @@ masked_conv_patch_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const
     const bool early_ok = a.fuse_compact && tid < WORK_THREADS && tid * 16 + 16 <= g.rows && (reinterpret_cast<uintptr_t>(a.mask) & 15) == 0;
     if (early_ok) early_mask = ptx::ld_global_v4_keep_in_l2(a.mask + tid * 16);
 
-    // barrier initialisation, one barrier per thread (a single thread took about 1500 clocks over them)
+    // barrier initialisation, one barrier per thread (a single thread took about 1500 clocks over them), by the
+    // block's last threads, so that warp 0's tensor-memory allocation runs beside it
     {
         constexpr int NB = FULL_RING + MAX_B_STAGES + MAX_A_STAGES + 2 * INFO_RING + 2 * MAX_P_BUFS + 4;
-        if (tid < NB) {
-            int i = tid;
+        if (tid >= NUM_THREADS - NB) {
+            int i = tid - (NUM_THREADS - NB);
             unsigned long long* bar;
             uint32_t count;
             if (i < FULL_RING) { bar = &sh->full[i]; count = 5; }                        // the filter thread's expect_tx + one arrival per lane quarter

@@ -177,24 +177,29 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
     const bool early_ok = a.fuse_compact && tid * 16 + 16 <= g.rows && (reinterpret_cast<uintptr_t>(a.mask) & 15) == 0;
     if (early_ok) early_mask = ptx::ld_global_v4_keep_in_l2(a.mask + tid * 16);
 
-    if (tid == 0) {
-        for (int s = 0; s < S; ++s) {
-            // the filter thread's expect_tx arrival (which in TMA mode also announces the gathered
+    // barrier initialisation, one barrier per thread (a single thread took about 1300 clocks over them); the
+    // threads are those of the last warps, so that the tensor-memory allocation of warp 1 runs beside it
+    {
+        constexpr int NB = 2 * MAX_STAGES + 2 * INFO_RING + 4;
+        int i = tid - (NUM_THREADS - NB);
+        if (i >= 0) {
+            unsigned long long* bar;
+            uint32_t count;
+            // full: the filter thread's expect_tx arrival (which in TMA mode also announces the gathered
             // bytes) + in the copy modes every gather lane's arrival
-            ptx::mbar_init(ptx::smem_u32(&sh->full[s]), 1 + (MODE == GATHER_TMA ? 0 : GROUP_WARPS * 32));
-            ptx::mbar_init(ptx::smem_u32(&sh->empty[s]), 1);
+            if (i < MAX_STAGES) { bar = &sh->full[i]; count = 1 + (MODE == GATHER_TMA ? 0 : GROUP_WARPS * 32); }
+            else if ((i -= MAX_STAGES) < MAX_STAGES) { bar = &sh->empty[i]; count = 1; }
+            else if ((i -= MAX_STAGES) < INFO_RING) { bar = &sh->info_full[i]; count = 1; }
+            else if ((i -= INFO_RING) < INFO_RING) { bar = &sh->info_empty[i]; count = NUM_PROD_WARPS; }    // one arrival per gather warp
+            else if ((i -= INFO_RING) < 2) { bar = &sh->acc_full[i]; count = 1; }
+            else { i -= 2; bar = &sh->acc_empty[i]; count = NUM_EPI_WARPS; }
+            ptx::mbar_init(ptx::smem_u32(bar), count);
+            ptx::fence_mbar_init();
         }
-        for (int i = 0; i < INFO_RING; ++i) {
-            ptx::mbar_init(ptx::smem_u32(&sh->info_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh->info_empty[i]), NUM_PROD_WARPS);  // one arrival per gather warp
+        if (tid == 0) {
+            sh->ctl.abort = 0;
+            sh->ctl.limit_kcycles = a.wait_limit_kcycles;
         }
-        for (int i = 0; i < 2; ++i) {
-            ptx::mbar_init(ptx::smem_u32(&sh->acc_full[i]), 1);
-            ptx::mbar_init(ptx::smem_u32(&sh->acc_empty[i]), NUM_EPI_WARPS);
-        }
-        sh->ctl.abort = 0;
-        sh->ctl.limit_kcycles = a.wait_limit_kcycles;
-        ptx::fence_mbar_init();
     }
     if (warp == WARP_MMA) {
         ptx::tmem_alloc(ptx::smem_u32(&sh->tmem_base), (uint32_t)a.tmem_cols);
