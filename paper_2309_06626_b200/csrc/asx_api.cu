@@ -524,8 +524,7 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
             L->tmap_ptr = nullptr;
             L->tmapx_ptr = nullptr;
         }
-        cudaError_t e = launch_stage_blocks2x2(x, L->d_xpad, Nb, H, W, L->C_in, Hs, Ws, h0, st);
-        if (e == cudaSuccess) e = launch_pack_block_filters(w, L->d_wpack, L->C_out, L->kh, L->kw, L->C_in, kh2, bshift, st);
+        cudaError_t e = launch_stage_blocks2x2(x, L->d_xpad, Nb, H, W, L->C_in, Hs, Ws, h0, w, L->d_wpack, L->C_out, L->kh, L->kw, kh2, bshift, st);
         if (e != cudaSuccess) return from_cuda(e);
         xsrc = L->d_xpad;
         wsrc = L->d_wpack;

@@ -109,10 +109,9 @@ cudaError_t launch_pad_channels(const void* src, void* dst, long long rows, int 
 // filters for the pixel-pair form: w[C_out][kh][kw][C] -> w2[C_out][kh][kw2][2][4], where pair kxx,
 // half j holds the original tap kx = 2*kxx + j - shift (zero when outside 0..kw-1 or c >= C)
 cudaError_t launch_mask_from_activation(const void* x, long long rows, int C, uint8_t* mask, int num_sms, cudaStream_t st);
+// 2x2-block form of a first layer: the staged input (xs) and the packed filters (w2), one launch
 cudaError_t launch_stage_blocks2x2(const void* x, void* xs, int Nb, int H, int W, int C, int Hs, int Ws, int h0,
-                                   cudaStream_t st);
-cudaError_t launch_pack_block_filters(const void* w, void* w2, int C_out, int kh, int kw, int C, int kh2, int shift,
-                                      cudaStream_t st);
+                                   const void* w, void* w2, int C_out, int kh, int kw, int kh2, int shift, cudaStream_t st);
 cudaError_t launch_pack_pair_filters(const void* w, void* w2, int C_out, int kh, int kw, int C, int kw2, int shift,
                                      cudaStream_t st);
 

@@ -775,22 +775,43 @@ __global__ void pack_pair_filters_kernel(const unsigned short* __restrict__ w, u
     }
 }
 
+// Filters of the 2x2-block form: w2[co][ky2][kx2][r][px][4] = w[co][2 ky2 + r - shift][2 kx2 + px - shift][c],
+// zero outside the filter and for c >= C.  kx2 runs over 4 blocks (one 128-byte run of the input per
+// filter block row).  One thread per output element, `nthreads` threads of which this is number `t`.
+__device__ __forceinline__ void pack_block_filters(const unsigned short* __restrict__ w, unsigned short* __restrict__ w2,
+                                                   int C_out, int kh, int kw, int C, int kh2, int shift, int t, int nthreads)
+{
+    const int total = C_out * kh2 * 64;
+    for (int i = t; i < total; i += nthreads) {
+        const int c = i & 3, px = (i >> 2) & 1, r = (i >> 3) & 1, kx2 = (i >> 4) & 3;
+        const int rest = i >> 6;
+        const int ky2 = rest % kh2, co = rest / kh2;
+        const int ky = 2 * ky2 + r - shift, kx = 2 * kx2 + px - shift;
+        w2[i] = (ky >= 0 && ky < kh && kx >= 0 && kx < kw && c < C) ? w[(((long long)co * kh + ky) * kw + kx) * C + c]
+                                                                     : (unsigned short)0;
+    }
+}
+
 // Input of the 2x2-block form (see asx_run): xs[n][ys][xs][r][px][4] holds the 2x2 pixel block
 // whose top-left pixel is (2 (ys - h0), 2 (xs - h0)), channels padded to 4, zeros outside the image.
-// One thread per block (32 bytes).
-__global__ void stage_blocks2x2_kernel(const unsigned short* __restrict__ x, uint4* __restrict__ xs, int Nb, int H, int W,
-                                       int C, int Hs, int Ws, int h0)
+// Block (ys, n) of the grid writes one staged row, one thread per 2x2 block (32 bytes), so that nothing
+// divides; the blocks with n = Nb pack the filters instead (the same launch does both).
+__global__ void __launch_bounds__(128) stage_blocks2x2_kernel(const unsigned short* __restrict__ x, uint4* __restrict__ xs, int Nb, int H, int W,
+                                                              int C, int Hs, int Ws, int h0, const unsigned short* __restrict__ w,
+                                                              unsigned short* __restrict__ w2, int C_out, int kh, int kw, int kh2, int shift)
 {
     ptx::grid_launch_dependents();
     ptx::grid_dependency_wait();
-    const long long total = (long long)Nb * Hs * Ws;
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
-         i += (long long)gridDim.x * blockDim.x) {
-        const int bx = (int)(i % Ws);
-        const long long rest = i / Ws;
-        const int by = (int)(rest % Hs), n = (int)(rest / Hs);
+    const int by = blockIdx.x, n = blockIdx.y;
+    if (n == Nb) {
+        pack_block_filters(w, w2, C_out, kh, kw, C, kh2, shift, by * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
+        return;
+    }
+    const long long row0 = ((long long)n * Hs + by) * Ws;
+    const bool words = (C == 3 && (reinterpret_cast<uintptr_t>(x) & 3) == 0);
+    for (int bx = threadIdx.x; bx < Ws; bx += blockDim.x) {
         unsigned short v[16];
-        if (C == 3 && (reinterpret_cast<uintptr_t>(x) & 3) == 0) {
+        if (words) {
             // three channels: the two pixels of a block row are 12 contiguous bytes at a 4-byte
             // aligned offset (the block's first column is even), i.e. three 32-bit loads
 #pragma unroll
@@ -807,44 +828,25 @@ __global__ void stage_blocks2x2_kernel(const unsigned short* __restrict__ x, uin
                 v[r * 8 + 4] = (unsigned short)(q1 >> 16);     v[r * 8 + 5] = (unsigned short)(q2 & 0xffffu);
                 v[r * 8 + 6] = (unsigned short)(q2 >> 16);     v[r * 8 + 7] = 0;
             }
-        } else
+        } else {
 #pragma unroll
-        for (int r = 0; r < 2; ++r)
+            for (int r = 0; r < 2; ++r)
 #pragma unroll
-            for (int px = 0; px < 2; ++px) {
-                const int iy = 2 * (by - h0) + r, ix = 2 * (bx - h0) + px;
-                const bool in = iy >= 0 && iy < H && ix >= 0 && ix < W;
-                const unsigned short* src = x + (((long long)n * H + (in ? iy : 0)) * W + (in ? ix : 0)) * C;
+                for (int px = 0; px < 2; ++px) {
+                    const int iy = 2 * (by - h0) + r, ix = 2 * (bx - h0) + px;
+                    const bool in = iy >= 0 && iy < H && ix >= 0 && ix < W;
+                    const unsigned short* src = x + (((long long)n * H + (in ? iy : 0)) * W + (in ? ix : 0)) * C;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) v[(r * 2 + px) * 4 + c] = (in && c < C) ? __ldcg(src + c) : (unsigned short)0;
-            }
+                    for (int c = 0; c < 4; ++c) v[(r * 2 + px) * 4 + c] = (in && c < C) ? __ldcg(src + c) : (unsigned short)0;
+                }
+        }
         uint4 lo, hi;
         lo.x = v[0] | ((uint32_t)v[1] << 16); lo.y = v[2] | ((uint32_t)v[3] << 16);
         lo.z = v[4] | ((uint32_t)v[5] << 16); lo.w = v[6] | ((uint32_t)v[7] << 16);
         hi.x = v[8] | ((uint32_t)v[9] << 16); hi.y = v[10] | ((uint32_t)v[11] << 16);
         hi.z = v[12] | ((uint32_t)v[13] << 16); hi.w = v[14] | ((uint32_t)v[15] << 16);
-        xs[2 * i] = lo;
-        xs[2 * i + 1] = hi;
-    }
-}
-
-// Filters of the 2x2-block form: w2[co][ky2][kx2][r][px][4] = w[co][2 ky2 + r - shift][2 kx2 + px - shift][c],
-// zero outside the filter and for c >= C.  kx2 runs over 4 blocks (one 128-byte run of the input per
-// filter block row).  One thread per output element.
-__global__ void pack_block_filters_kernel(const unsigned short* __restrict__ w, unsigned short* __restrict__ w2,
-                                          int C_out, int kh, int kw, int C, int kh2, int shift)
-{
-    ptx::grid_launch_dependents();
-    ptx::grid_dependency_wait();
-    const long long total = (long long)C_out * kh2 * 64;
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
-         i += (long long)gridDim.x * blockDim.x) {
-        const int c = (int)(i & 3), px = (int)((i >> 2) & 1), r = (int)((i >> 3) & 1), kx2 = (int)((i >> 4) & 3);
-        const long long rest = i >> 6;
-        const int ky2 = (int)(rest % kh2), co = (int)(rest / kh2);
-        const int ky = 2 * ky2 + r - shift, kx = 2 * kx2 + px - shift;
-        w2[i] = (ky >= 0 && ky < kh && kx >= 0 && kx < kw && c < C) ? w[(((long long)co * kh + ky) * kw + kx) * C + c]
-                                                                     : (unsigned short)0;
+        xs[2 * (row0 + bx)] = lo;
+        xs[2 * (row0 + bx) + 1] = hi;
     }
 }
 
@@ -1004,23 +1006,12 @@ cudaError_t launch_pack_pair_filters(const void* w, void* w2, int C_out, int kh,
 }
 
 cudaError_t launch_stage_blocks2x2(const void* x, void* xs, int Nb, int H, int W, int C, int Hs, int Ws, int h0,
-                                   cudaStream_t st)
+                                   const void* w, void* w2, int C_out, int kh, int kw, int kh2, int shift, cudaStream_t st)
 {
-    const long long total = (long long)Nb * Hs * Ws;
-    int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
-    if (blocks < 1) blocks = 1;
-    return launch_pdl(stage_blocks2x2_kernel, dim3(blocks), dim3(256), 0, st, static_cast<const unsigned short*>(x),
-                      static_cast<uint4*>(xs), Nb, H, W, C, Hs, Ws, h0);
-}
-
-cudaError_t launch_pack_block_filters(const void* w, void* w2, int C_out, int kh, int kw, int C, int kh2, int shift,
-                                      cudaStream_t st)
-{
-    const long long total = (long long)C_out * kh2 * 64;
-    int blocks = (int)((total + 255) / 256 < 1024 ? (total + 255) / 256 : 1024);
-    if (blocks < 1) blocks = 1;
-    return launch_pdl(pack_block_filters_kernel, dim3(blocks), dim3(256), 0, st, static_cast<const unsigned short*>(w),
-                      static_cast<unsigned short*>(w2), C_out, kh, kw, C, kh2, shift);
+    if (Hs < 1 || Nb < 1 || Nb >= 65535 || (long long)C_out * kh2 * 64 >= (1ll << 31)) return cudaErrorInvalidValue;
+    return launch_pdl(stage_blocks2x2_kernel, dim3(Hs, Nb + 1), dim3(128), 0, st, static_cast<const unsigned short*>(x),
+                      static_cast<uint4*>(xs), Nb, H, W, C, Hs, Ws, h0, static_cast<const unsigned short*>(w),
+                      static_cast<unsigned short*>(w2), C_out, kh, kw, kh2, shift);
 }
 
 }  // namespace asx
