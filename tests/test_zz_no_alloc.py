@@ -67,7 +67,7 @@ def test_static_compaction_rejects_sizes_beyond_its_scratch():
 
 @pytest.mark.parametrize("rows", [0, 1, 16384, 16385, COMPACT_STATIC_MAX_ROWS])
 def test_static_compaction_sizes_at_the_edges_of_its_two_forms(rows):
-    """No rows, one row, the largest mask the one-block form takes, the smallest the three passes take,
+    """No rows, one row, the largest mask the one-block form takes, the smallest the two passes take,
     and the largest the built-in scratch holds (every word of it in use)."""
     rng = np.random.default_rng(rows + 3)
     m = (rng.random(rows) < 0.37).astype(np.uint8)
