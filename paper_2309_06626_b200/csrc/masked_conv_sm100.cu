@@ -809,6 +809,30 @@ __global__ void __launch_bounds__(128) stage_blocks2x2_kernel(const unsigned sho
     }
     const long long row0 = ((long long)n * Hs + by) * Ws;
     const bool words = (C == 3 && (reinterpret_cast<uintptr_t>(x) & 3) == 0);
+    if (words && (reinterpret_cast<uintptr_t>(x) & 7) == 0 && (h0 & 1) == 0 && (W & 3) == 0 && (Ws & 1) == 0) {
+        // three channels, two blocks per thread: the four pixels of a block-row pair are 24 contiguous bytes at an
+        // 8-byte aligned offset (first column a multiple of 4, W a multiple of 4), i.e. three 64-bit loads per image row
+        for (int bp = threadIdx.x; 2 * bp < Ws; bp += blockDim.x) {
+            const int bx = 2 * bp;
+            uint4 o[2][2];                      // [block][image row]
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int iy = 2 * (by - h0) + r, ix = 2 * (bx - h0);
+                const bool in = iy >= 0 && iy < H && ix >= 0 && ix < W;       // ix and W are multiples of 4: all four pixels or none
+                uint2 q0 = make_uint2(0, 0), q1 = q0, q2 = q0;
+                if (in) {
+                    const uint2* src = reinterpret_cast<const uint2*>(x + (((long long)n * H + iy) * W + ix) * 3);
+                    q0 = __ldcg(src); q1 = __ldcg(src + 1); q2 = __ldcg(src + 2);
+                }
+                // 12 values p0c0 p0c1 p0c2 p1c0 | p1c1 p1c2 p2c0 p2c1 | p2c2 p3c0 p3c1 p3c2 -> two blocks of (px0 c0..2 0, px1 c0..2 0)
+                o[0][r] = make_uint4(q0.x, q0.y & 0xffffu, (q0.y >> 16) | (q1.x << 16), q1.x >> 16);
+                o[1][r] = make_uint4(q1.y, q2.x & 0xffffu, (q2.x >> 16) | (q2.y << 16), q2.y >> 16);
+            }
+            uint4* dst = xs + 2 * (row0 + bx);
+            dst[0] = o[0][0]; dst[1] = o[0][1]; dst[2] = o[1][0]; dst[3] = o[1][1];
+        }
+        return;
+    }
     for (int bx = threadIdx.x; bx < Ws; bx += blockDim.x) {
         unsigned short v[16];
         if (words) {
