@@ -37,11 +37,11 @@ L2_BYTES = 126 * 1024 * 1024
 
 # DRAM traffic of the fused kernels from one ncu capture of the default workload (ResNet-18 stack, batch 64):
 # dram__bytes_read.sum + dram__bytes_write.sum averaged over the 20 fused-kernel launches of a step
-# (12.79 MB read + 2.36 MB written; ncu flushes the caches before every captured launch, so reads are
+# (12.79 MB read + 2.35 MB written; ncu flushes the caches before every captured launch, so reads are
 # cold-cache and most of a launch's output is still in L2 when its counters stop).  The figure belongs to
 # the kernel sources whose digest is recorded with it; with any other sources the bench reports null.
-NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 15.15e6,
-               "csrc_sha256": "2a3a3ac69e780e84bc0b84fba4324daa4ab2b17054028156cb3977be936f60e5"}
+NCU_TRAFFIC = {"workload_config": 3, "bytes_per_launch": 15.14e6,
+               "csrc_sha256": "59b86307211c318abd38b581461edbda71f1d77579a3bb243d1ee5c672f483ef"}
 
 
 def csrc_digest() -> str:
