@@ -268,14 +268,14 @@ class DeviceLayer:
         self.bytes = wl.algorithmic_bytes(spec, self.mask, 4 if f32 else 2)
         self.ptrs = (self.x.data_ptr(), spec.Nb, spec.H, spec.W, self.w.data_ptr(), self.b.data_ptr(),
                      self.y.data_ptr())
-        # fused kernel (it rebuilds the kept-row list itself for masks of up to 16384 rows, else the two
+        # fused kernel (it rebuilds the kept-row list itself for masks of up to 32768 rows, else the two
         # compaction passes run first), plus the staging of x and w when C_in is not a multiple of 8 (4 in fp32):
         # one launch in the 2x2-block form of a stride-2 first layer, else one padding launch each
         sh = spec.pad & 1
         blocks2x2 = (not f32 and spec.C_in <= 4 and spec.stride == 2 and spec.W % 2 == 0 and spec.H % 2 == 0
                      and (spec.kw + sh + 1) // 2 == 4 and spec.kh + sh <= 32)
         staging = 1 if blocks2x2 else (2 if spec.C_in % (4 if f32 else 8) else 0)
-        self.launches = 1 + (0 if self.mask.size <= 16384 else 2) + staging
+        self.launches = 1 + (0 if self.mask.size <= 32768 else 2) + staging
 
     def step(self, st, flags, layer=None, recompact=True):
         L = layer or self.layer
@@ -753,7 +753,7 @@ def run_ours(args):
                    "l2": f"inputs larger than L2: each step cycles {footprint / 1e6:.0f} MB of distinct "
                          f"layer buffers (L2 is {L2_BYTES / 1e6:.0f} MB)",
                    "step": "per layer: one asx_run with ASX_RECOMPACT = mask compaction (inside the fused kernel "
-                           "for masks <= 16384 rows) + gather/GEMM/scatter"
+                           "for masks <= 32768 rows) + gather/GEMM/scatter"
                            + ("" if graph is None else "; one step = one CUDA-graph replay")
                            + ("; the 1x1 projection of each down-sampling block runs on a graph branch beside that block's "
                               "conv1 -> conv2, as in the network" if (fork and graph is not None) else ""),

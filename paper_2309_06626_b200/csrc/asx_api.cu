@@ -465,10 +465,11 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     L->last_stream = st;
-    // Small masks are compacted inside the fused kernel itself (one launch instead of two); the
-    // reference kernel and large masks take the stand-alone compaction kernel.
-    const bool fuse_compact = (flags & ASX_RECOMPACT) && !(flags & ASX_IMPL_NAIVE) &&
-                              L->rows <= COMPACT_SMALL_MAX_ROWS;
+    // Small masks are compacted inside the fused kernel itself (no launches of its own, and the list stays in
+    // shared memory as 16-bit positions); the reference kernel and large masks take the stand-alone compaction
+    // kernels.  Up to 16384 rows always; up to FUSED_COMPACT_MAX_ROWS when the list (2 bytes per row) still
+    // leaves the plan its pipeline stages (decided below, once the geometry the kernel sees is known).
+    bool fuse_compact = (flags & ASX_RECOMPACT) && !(flags & ASX_IMPL_NAIVE) && L->rows <= FUSED_COMPACT_MAX_ROWS;
     if ((flags & ASX_RECOMPACT) && !fuse_compact) {
         s = run_compaction(L, st);
         if (s != ASX_OK) return s;
@@ -620,7 +621,14 @@ asx_status asx_run(asx_layer* L, const void* x, int Nb, int H, int W, const void
     // Sharing a tile's k-blocks between blocks needs the exact tile count (to size the workspace)
     // and 16-byte output stores.
     const bool allow_split = !f32 && L->host_kept >= 0 && L->C_out % 8 == 0 && (reinterpret_cast<uintptr_t>(y) & 15) == 0;
-    if (!plan_fast(g, L->num_sms, est_rows, fuse_compact ? (int)L->rows : 0, allow_split, ES, &plan)) return ASX_ERR_UNSUPPORTED;
+    if (!plan_fast(g, L->num_sms, est_rows, fuse_compact ? (int)L->rows : 0, allow_split, ES, &plan)) {
+        if (!(fuse_compact && L->rows > COMPACT_SMALL_MAX_ROWS)) return ASX_ERR_UNSUPPORTED;
+        // no room for the list beside the pipeline stages: the stand-alone compaction, and the list in global memory
+        fuse_compact = false;
+        s = run_compaction(L, st);
+        if (s != ASX_OK) return s;
+        if (!plan_fast(g, L->num_sms, est_rows, 0, allow_split, ES, &plan)) return ASX_ERR_UNSUPPORTED;
+    }
     // Stride-1 layers with several filter taps and whole 64-channel slices take the window-patch form
     // when the host knows the mask, every tile's windows fit the patch buffers and the planner's
     // estimate favours it; compact inputs and fp32 storage stay with the row gather.

@@ -43,6 +43,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 
 // ---- S1: mask compaction (compact.cu)
 constexpr int COMPACT_SMALL_MAX_ROWS = 1024 * 16;   // one block handles masks up to this size
+constexpr int FUSED_COMPACT_MAX_ROWS = 1024 * 32;   // the fused kernels rebuild lists of up to this many rows themselves (positions fit 16 bits)
 constexpr int COMPACT_THREADS = 256;
 constexpr int COMPACT_PER_THREAD = 16;
 constexpr int COMPACT_TILE = COMPACT_THREADS * COMPACT_PER_THREAD;

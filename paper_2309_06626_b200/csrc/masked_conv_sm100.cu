@@ -123,12 +123,11 @@ __device__ __forceinline__ Item item_of(int t, int KB, const FastArgs& a)
 // window's corner, (n H + iy0) W + ix0 (with a compact input: the first input row of its image,
 // n * in_kept), and the corner's coordinates packed as iy0 << 16 | ix0.
 // Rows past the end get iy0 = -32768, for which no filter tap is inside the image.
-__device__ __forceinline__ int2 row_info_of(int rk, int Mk, const FastDiv& fdcnt, const ConvGeom& g, const FastArgs& a,
-                                            const KeptList& kept)
+// (row: the output row of the kept row, as out_row_of gives it, or -1 past the end)
+__device__ __forceinline__ int2 row_info_from_row(int row, const ConvGeom& g, const FastArgs& a)
 {
     int2 info = make_int2(0, (int)0x80000000u);
-    if (rk < Mk) {
-        const int row = out_row_of(rk, fdcnt, g, kept);
+    if (row >= 0) {
         if (row < g.M) {
             const int n = (int)fd_div((uint32_t)row, a.fdP), p = row - n * g.P;
             const int oy = (int)fd_div((uint32_t)p, a.fdWo), ox = p - oy * g.Wo;
@@ -140,6 +139,11 @@ __device__ __forceinline__ int2 row_info_of(int rk, int Mk, const FastDiv& fdcnt
         }
     }
     return info;
+}
+__device__ __forceinline__ int2 row_info_of(int rk, int Mk, const FastDiv& fdcnt, const ConvGeom& g, const FastArgs& a,
+                                            const KeptList& kept)
+{
+    return row_info_from_row(rk < Mk ? out_row_of(rk, fdcnt, g, kept) : -1, g, a);
 }
 
 // SILU: the activation is z / (1 + exp(-z)) instead of the run-time choice between ReLU and identity
@@ -295,11 +299,17 @@ masked_conv_sm100_kernel(const __grid_constant__ CUtensorMap tmap_w, const __gri
             good = __shfl_sync(0xffffffffu, good, 0);
             if (!good) break;
             const int m_tile = item_of((int)t, KB, a).m_tile;
+            // the four list entries first (with the list in global memory each is a trip to L2: one after the other
+            // they were 2.7 us per tile, which paced every layer with one k-block per tile and a mask too large for
+            // the fused compaction), then the arithmetic
+            int rows4[4];
 #pragma unroll
             for (int q2 = 0; q2 < 4; ++q2) {
-                const int rr = lane * 4 + q2;
-                sh->rowinfo[r][rr] = row_info_of(m_tile * BM + rr, Mk, fdcnt, g, a, kept_list);
+                const int rk = m_tile * BM + lane * 4 + q2;
+                rows4[q2] = rk < Mk ? out_row_of(rk, fdcnt, g, kept_list) : -1;
             }
+#pragma unroll
+            for (int q2 = 0; q2 < 4; ++q2) sh->rowinfo[r][lane * 4 + q2] = row_info_from_row(rows4[q2], g, a);
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&sh->info_full[r]));
         }
