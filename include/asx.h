@@ -267,8 +267,9 @@ asx_status asx_destroy(asx_layer* layer);
  *               bytes, 8-byte aligned; contents on entry are irrelevant (every word that is
  *               read is written first, in stream order).  Calls sharing one scratch buffer
  *               must not overlap.
- * Masks of more than 16384 rows take three launches (tile counts, their scan, the ordered
- * write; the mask is read twice), smaller ones a single block; no block waits for another.
+ * Masks of more than 16384 rows take two launches (kept rows counted per run of tiles, then the
+ * ordered write, in which every block sums the counts in front of its run; the mask is read
+ * twice), smaller ones a single block; no block waits for another.
  * 0 <= rows < 2^31.  Asynchronous on `cuda_stream`; allocates nothing.
  */
 int64_t asx_compact_scratch_bytes(int64_t rows);
