@@ -5,6 +5,8 @@ import torch
 
 import oracle
 import paper_2309_06626_b200 as asx
+import workloads as wl
+from gpu_util import make_problem, max_abs_tol, to_dev_bf16, REL_FROB_TOL
 
 pytestmark = pytest.mark.gpu
 
@@ -31,9 +33,9 @@ def test_compaction_matches_oracle(rows, q):
 
 
 @pytest.mark.parametrize("rows", [16383, 16384, 16385, 16400, 32768, 32769, 16384 * 9 + 4095])
-def test_tile_boundaries_of_the_three_pass_form(rows):
+def test_tile_boundaries_of_the_two_pass_form(rows):
     """Row counts around the 16384-row tiles of the large-mask passes (one block up to 16384 rows,
-    count / scan / write above), with ragged and exactly full last tiles."""
+    count / write by resident blocks above), with ragged and exactly full last tiles."""
     rng = np.random.default_rng(rows)
     for q in (0.0, 0.37, 1.0):
         mask = (rng.random(rows) < q).astype(np.uint8)
@@ -41,9 +43,9 @@ def test_tile_boundaries_of_the_three_pass_form(rows):
         assert np.array_equal(kept, oracle.kept_list(mask))
 
 
-def test_more_tiles_than_one_round_of_the_tile_scan():
-    """2^27 rows and a bit: 8196 tiles, so the one-block scan of the tile counts (8192 per round)
-    carries a running total into a second round; kept runs that straddle tile boundaries."""
+def test_more_tiles_than_resident_blocks():
+    """2^27 rows and a bit: 8196 tiles on 1184 resident blocks, so every block walks a run of tiles and
+    sums a thousand run counts for its offset; kept runs that straddle tile and run boundaries."""
     rows = (1 << 27) + 3 * 16384 + 5
     rng = np.random.default_rng(27)
     mask = (rng.random(rows) < 0.5).astype(np.uint8)
@@ -128,3 +130,39 @@ def test_mask_written_by_the_kernel_just_before(rows):
         assert int(c1.item()) == want.size and int(c2.item()) == want.size, r
         assert np.array_equal(k1[:want.size].cpu().numpy(), want), r
         assert np.array_equal(k2[:want.size].cpu().numpy(), want), r
+
+
+@pytest.mark.parametrize("case", [
+    # name, C_in, C_out, k, pad, H, W, Nb, pct, block, fused list expected to fit beside the pipeline stages
+    ("pw_160", 32, 32, 1, 0, 160, 160, 1, 40, 4),              # 25600-row mask: compacted inside the fused kernel
+    ("pw_181x181", 64, 64, 1, 0, 181, 181, 1, 50, 1),          # 32761 rows: just under the limit
+    ("pw_182x182", 64, 64, 1, 0, 182, 182, 1, 50, 1),          # 33124 rows: the stand-alone passes
+    ("c3_150_wide", 64, 256, 3, 1, 150, 150, 1, 70, 2),        # 22500 rows, 256-wide tiles: no room for the list, falls back
+], ids=lambda c: c[0])
+def test_masks_between_the_one_block_limit_and_the_fused_limit(case):
+    """Masks of 16385..32768 rows are compacted inside the fused kernel when their 2-byte list fits beside the
+    pipeline stages, by the stand-alone passes otherwise; either way ASX_RECOMPACT must give the stored list's result
+    and the oracle's."""
+    name, cin, cout, k, pad, H, W, Nb, pct, blk = case
+    spec = wl.LayerSpec(name, cin, cout, k, k, 1, pad, H, W, Nb, pct, blk, "relu", wl.BASE_SEED + 8800 + H)
+    x, w, b, mask = make_problem(spec, per_row=False)
+    layer = asx.MaskedConvLayer(cin, cout, k, k, 1, pad)
+    layer.set_mask(mask)
+    xd, wd, bd = to_dev_bf16(x), to_dev_bf16(w), torch.from_numpy(b).cuda()
+    y_stored = layer.run(xd, wd, bd, flags=asx.ACT_RELU).clone()
+    y_re = layer.run(xd, wd, bd, flags=asx.ACT_RELU | asx.RECOMPACT).clone()
+    torch.cuda.synchronize()
+    assert layer.device_status() == 0
+    assert np.array_equal(layer.kept(), oracle.kept_list(mask))
+    assert torch.equal(y_stored.view(torch.int16), y_re.view(torch.int16))
+    # a new mask through the device copy only (no host-side list): the next RECOMPACT run must follow it
+    mask2 = np.roll(mask, 7)
+    layer.set_mask(mask2)
+    y2 = layer.run(xd, wd, bd, flags=asx.ACT_RELU | asx.RECOMPACT)
+    torch.cuda.synchronize()
+    assert np.array_equal(layer.kept(), oracle.kept_list(mask2))
+    ref = oracle.masked_conv(x, w, b, mask2, 1, pad, True).reshape(spec.M, cout)
+    got = y2.float().cpu().numpy().astype(np.float64).reshape(spec.M, cout)
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= REL_FROB_TOL
+    assert np.abs(got - ref).max() <= max_abs_tol(spec.K, oracle.bf16_round(x), oracle.bf16_round(w))
+    layer.close()
